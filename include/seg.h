@@ -1,0 +1,204 @@
+/*
+ * seg.h - C ABI of the segment trainer: one independently trained, fully connected
+ * network segment with synthetic intermediate labels (SIL), on one NVIDIA B200 (sm_100a).
+ *
+ * Method: "Partitioned Neural Network Training via Synthetic Intermediate Labels".
+ * A network is cut into consecutive segments.  Each cut gets one random target vector
+ * per class (Eq. 1); a non-final segment is trained to map its input to the target
+ * vector of the sample's class, the final segment is trained on the class labels
+ * (Section 2).  Segments never exchange activations or gradients while training
+ * (Section 1), so one handle holds everything a segment needs.
+ *
+ * Conventions
+ *   - All tensor arguments are DEVICE pointers unless a comment says "host".
+ *   - Matrices are row-major and dense (pitch = number of columns) at this boundary.
+ *   - A Linear layer l computes Z = A_prev * W^T + b with W stored [out][in].
+ *   - Every call enqueues its work on the stream given at seg_create and returns
+ *     without synchronising.  The caller keeps argument buffers alive and unchanged
+ *     until the stream has consumed them.
+ *   - Argument errors are reported synchronously through the return code and enqueue
+ *     nothing.  Device-side problems (a bounded wait that ran out) are recorded in a
+ *     status word that seg_poll_status reads.
+ *   - Nothing is thrown across this boundary and nothing aborts the process.
+ *   - A handle is not thread-safe; different handles may be used from different
+ *     threads and on different streams concurrently.
+ */
+#ifndef SEG_H_
+#define SEG_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SEG_API __attribute__((visibility("default")))
+#else
+#define SEG_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct seg_handle seg_handle; /* opaque, owned by the library */
+
+typedef enum {
+  SEG_OK = 0,
+  SEG_ERR_INVALID_ARG = 1,    /* null pointer, value out of range                      */
+  SEG_ERR_SHAPE = 2,          /* batch > max_batch, layer index out of range, ...      */
+  SEG_ERR_UNSUPPORTED = 3,    /* combination the library does not implement            */
+  SEG_ERR_ALLOC = 4,          /* device allocation failed                              */
+  SEG_ERR_CUDA = 5,           /* a CUDA runtime or driver call failed                  */
+  SEG_ERR_STATE = 6,          /* call order: e.g. training on labels never generated   */
+  SEG_ERR_DEVICE_TIMEOUT = 7, /* a kernel gave up a bounded wait and returned early    */
+  SEG_ERR_NO_DEVICE = 8       /* no CUDA device / not an sm_100 device                 */
+} seg_status;
+
+/* Arithmetic of the matrix products.  Accumulation is always fp32.
+ *   SEG_FP32: fp32 operands (FFMA).               x, y are float.
+ *   SEG_TF32: fp32 storage, operands rounded to TF32 (nearest even) where they are
+ *             stored: weights in a rounded copy, activations and dZ on store.  x, y float.
+ *   SEG_BF16: fp32 master weights with a bf16 copy, bf16 activations and dZ.
+ *             x and the y of a non-final segment are bf16 (raw 16-bit patterns);
+ *             the logits of a final segment are float.                                    */
+typedef enum { SEG_FP32 = 0, SEG_TF32 = 1, SEG_BF16 = 2 } seg_precision;
+
+/* Section 3 uses SGD with momentum 0.9; plain SGD and Adam serve the synthetic workloads.
+ *   SEG_SGD:          p -= lr * g
+ *   SEG_SGD_MOMENTUM: buf = momentum * buf + g;  p -= lr * buf        (buf starts at 0)
+ *   SEG_ADAM:         m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2;
+ *                     p -= lr * (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps),  t = 1, 2, ... */
+typedef enum { SEG_SGD = 0, SEG_SGD_MOMENTUM = 1, SEG_ADAM = 2 } seg_optimizer;
+
+/* Distribution of the intermediate labels.
+ *   SEG_LABEL_UNIFORM_KAPPA: Eq. 1, SIL_ij ~ kappa * U(0,1) (Section 3 uses kappa = 10).
+ *   SEG_LABEL_NORMAL:        N(0,1) targets (the synthetic workloads); kappa is ignored.  */
+typedef enum { SEG_LABEL_UNIFORM_KAPPA = 0, SEG_LABEL_NORMAL = 1 } seg_label_dist;
+
+/* Which matrix-product kernels a handle uses. */
+typedef enum {
+  SEG_GEMM_AUTO = 0,   /* tensor cores for SEG_TF32 / SEG_BF16, FFMA for SEG_FP32 */
+  SEG_GEMM_SIMT = 1,   /* FFMA kernels for every precision (same rounding points)  */
+  SEG_GEMM_TCGEN05 = 2 /* tensor-core kernels; SEG_ERR_UNSUPPORTED with SEG_FP32   */
+} seg_gemm_backend;
+
+typedef struct {
+  int32_t n_layers;        /* Linear layers in this segment, 1..16 (Section 3: 2 and 3)   */
+  const int32_t* widths;   /* host; n_layers+1 entries: input width, then every layer's
+                              output width.  Copied by seg_create.                         */
+  int32_t n_classes;       /* M, the number of classes (Section 2)                         */
+  int32_t is_final;        /* 0: trained against SIL[class] with mean squared error;
+                              1: last segment, softmax cross-entropy on the class labels   */
+  int32_t last_relu;       /* ReLU on this segment's last layer: 1 / 0, or -1 for the
+                              default (1 if !is_final, 0 if is_final: Section 3 exempts
+                              only the network's final layer from ReLU)                    */
+  int32_t segment_id;      /* index of the segment / its cut; enters the random streams     */
+  int32_t precision;       /* seg_precision                                                */
+  int32_t optimizer;       /* seg_optimizer                                                */
+  float lr, momentum, beta1, beta2, eps;
+  int32_t max_batch;       /* workspaces are sized for this batch                          */
+  int32_t gemm_backend;    /* seg_gemm_backend                                             */
+  uint64_t init_seed;      /* seed of the weight-initialisation streams                    */
+  void* stream;            /* cudaStream_t every call of this handle enqueues on           */
+} seg_config;
+
+/* Creates a segment on the current device: allocates parameters, optimizer state,
+ * gradient, activation and dZ workspaces (all owned by the handle, freed by
+ * seg_destroy) and initialises W, b ~ U(-1/sqrt(fan_in), 1/sqrt(fan_in)) from Philox
+ * streams keyed by init_seed (Section 2 refers to the framework's default Linear
+ * initialisation).  cfg and out are host pointers.  On failure *out is NULL.             */
+SEG_API seg_status seg_create(const seg_config* cfg, seg_handle** out);
+
+/* Generates this segment's intermediate labels on the device (Eq. 1): an [M][N_P] fp32
+ * matrix, row j = target vector of class j (the paper's N_P x M matrix stored by
+ * columns), N_P = last width.  Element (j, i), flat index e = j*N_P+i, is word e mod 4 of
+ * the Philox4x32-10 block with key = (seed lo, seed hi) and counter
+ * (e/4 lo, e/4 hi, segment_id, 0); values are bit-reproducible on any device.  Valid for non-final segments only
+ * (SEG_ERR_STATE otherwise).                                                              */
+SEG_API seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, float kappa);
+
+/* One training step on one batch (Section 2: forward, loss against the intermediate
+ * target of each sample's class - or against the class label on the final segment -,
+ * backprop inside the segment, optimizer update).
+ *   x        [batch][widths[0]]  float (FP32/TF32) or bf16 (BF16)
+ *   cls      [batch] int32 class index in [0, M)
+ *   batch    1..max_batch
+ *   loss_out device float, receives the batch loss before the update; may be NULL
+ *   y_out    optional [batch][widths[n_layers]] copy of this step's forward output
+ *            (dtype as for seg_forward); may be NULL
+ * No gradient with respect to x is formed.                                                */
+SEG_API seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
+                          float* loss_out, void* y_out);
+
+/* The same step for callers whose batch lives in HOST memory: copies x_host and cls_host
+ * (host pointers; page-locked memory gives full copy speed) to device buffers the handle
+ * owns (allocated at the first such call), runs seg_train_step, copies the loss back to
+ * *loss_host (host float, may be NULL) and synchronises the stream before returning.     */
+SEG_API seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t* cls_host,
+                                       int32_t batch, float* loss_host);
+
+/* Forward pass only (the response handed to the next segment, Section 2):
+ *   y [batch][widths[n_layers]]: float for FP32/TF32 and for the logits of a final
+ *   segment, bf16 for a non-final BF16 segment.                                           */
+SEG_API seg_status seg_forward(seg_handle* h, const void* x, int32_t batch, void* y);
+
+/* Frees everything the handle owns.  Synchronises the handle's stream first.             */
+SEG_API seg_status seg_destroy(seg_handle* h);
+
+/* ---- auxiliary calls: inspection, injection, accounting ------------------------------ */
+
+/* Copies the [M][N_P] fp32 label matrix to / from a device buffer. */
+SEG_API seg_status seg_get_labels(seg_handle* h, float* dst);
+SEG_API seg_status seg_set_labels(seg_handle* h, const float* src);
+
+/* fp32 master parameters of layer `layer` (0-based): W [out][in], b [out]; either
+ * pointer may be NULL.  seg_set_params also refreshes the reduced-precision copy.        */
+SEG_API seg_status seg_get_params(seg_handle* h, int32_t layer, float* W, float* b);
+SEG_API seg_status seg_set_params(seg_handle* h, int32_t layer, const float* W, const float* b);
+
+/* Gradients of the last seg_train_step: dW [out][in], db [out], fp32. */
+SEG_API seg_status seg_get_grads(seg_handle* h, int32_t layer, float* dW, float* db);
+
+/* Optimizer state of layer `layer`: which = 0 momentum buffer / Adam first moment,
+ * which = 1 Adam second moment; shapes as the parameters.                                */
+SEG_API seg_status seg_get_opt_state(seg_handle* h, int32_t layer, int32_t which, float* sW, float* sb);
+
+/* Stored output A_layer of the last step, layer = 1..n_layers, converted to fp32
+ * [batch][widths[layer]] for the batch size of that step.                                */
+SEG_API seg_status seg_get_activation(seg_handle* h, int32_t layer, float* dst);
+
+/* Bytes of device memory the handle holds now and at its peak. host pointers. */
+SEG_API seg_status seg_mem_bytes(const seg_handle* h, uint64_t* current, uint64_t* peak);
+
+/* Number of kernels the handle has launched so far (host counter). */
+SEG_API seg_status seg_launch_count(const seg_handle* h, uint64_t* launches);
+
+/* Synchronises the handle's stream and returns SEG_ERR_DEVICE_TIMEOUT if any kernel of
+ * this handle gave up a bounded wait since the last poll, SEG_ERR_CUDA on a CUDA error.  */
+SEG_API seg_status seg_poll_status(seg_handle* h);
+
+/* Timing hooks: seg_timer_start / seg_timer_stop record CUDA events on the handle's
+ * stream; seg_timer_elapsed_ms synchronises on the stop event (host float out).          */
+SEG_API seg_status seg_timer_start(seg_handle* h);
+SEG_API seg_status seg_timer_stop(seg_handle* h);
+SEG_API seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms);
+
+/* Per-kernel timing (off by default).  While enabled, every launch of this handle is
+ * bracketed by CUDA events on the handle's stream.  seg_profile_get synchronises and
+ * returns, for one kernel kind, the number of launches and their summed device time
+ * since profiling was enabled; kinds: 0 forward product, 1 dgrad product, 2 wgrad
+ * product, 3 loss, 4 bias gradient, 5 optimizer update, 6 copies / staging.  count and
+ * total_ms are host pointers.                                                            */
+SEG_API seg_status seg_profile_enable(seg_handle* h, int32_t on);
+SEG_API seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms);
+
+SEG_API const char* seg_status_string(int32_t s);
+
+/* Text of the last CUDA error seen by this handle ("" if none); valid until the next call. */
+SEG_API const char* seg_last_error(const seg_handle* h);
+
+/* Static description of the build: "sm_100a ..." */
+SEG_API const char* seg_build_info(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEG_H_ */

@@ -1,0 +1,245 @@
+"""ctypes binding of libsegtrain.so: the functions of include/seg.h under the same names,
+plus `Segment`, a thin holder that marshals torch tensors into those calls.
+
+Argument marshalling only: every step of the training path runs in the library's CUDA
+kernels.  Importing this module without the built library raises; there is no CPU path.
+"""
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int32, c_uint64, c_void_p
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsegtrain.so")
+
+SEG_OK = 0
+SEG_FP32, SEG_TF32, SEG_BF16 = 0, 1, 2
+SEG_SGD, SEG_SGD_MOMENTUM, SEG_ADAM = 0, 1, 2
+SEG_LABEL_UNIFORM_KAPPA, SEG_LABEL_NORMAL = 0, 1
+SEG_GEMM_AUTO, SEG_GEMM_SIMT, SEG_GEMM_TCGEN05 = 0, 1, 2
+PRECISIONS = {"fp32": SEG_FP32, "tf32": SEG_TF32, "bf16": SEG_BF16}
+OPTIMIZERS = {"sgd": SEG_SGD, "momentum": SEG_SGD_MOMENTUM, "adam": SEG_ADAM}
+LABEL_DISTS = {"uniform_kappa": SEG_LABEL_UNIFORM_KAPPA, "normal": SEG_LABEL_NORMAL}
+BACKENDS = {"auto": SEG_GEMM_AUTO, "simt": SEG_GEMM_SIMT, "tcgen05": SEG_GEMM_TCGEN05}
+KERNEL_KINDS = ["fwd_gemm", "dgrad_gemm", "wgrad_gemm", "loss", "bias_grad", "update", "copy"]
+
+
+class seg_config(Structure):
+    _fields_ = [("n_layers", c_int32), ("widths", POINTER(c_int32)), ("n_classes", c_int32),
+                ("is_final", c_int32), ("last_relu", c_int32), ("segment_id", c_int32),
+                ("precision", c_int32), ("optimizer", c_int32),
+                ("lr", c_float), ("momentum", c_float), ("beta1", c_float), ("beta2", c_float),
+                ("eps", c_float), ("max_batch", c_int32), ("gemm_backend", c_int32),
+                ("init_seed", c_uint64), ("stream", c_void_p)]
+
+
+EXPORTS = {
+    "seg_create": (c_int32, [POINTER(seg_config), POINTER(c_void_p)]),
+    "seg_gen_labels": (c_int32, [c_void_p, c_uint64, c_int32, c_float]),
+    "seg_train_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
+    "seg_train_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_float)]),
+    "seg_forward": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p]),
+    "seg_destroy": (c_int32, [c_void_p]),
+    "seg_get_labels": (c_int32, [c_void_p, c_void_p]),
+    "seg_set_labels": (c_int32, [c_void_p, c_void_p]),
+    "seg_get_params": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p]),
+    "seg_set_params": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p]),
+    "seg_get_grads": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p]),
+    "seg_get_opt_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
+    "seg_get_activation": (c_int32, [c_void_p, c_int32, c_void_p]),
+    "seg_mem_bytes": (c_int32, [c_void_p, POINTER(c_uint64), POINTER(c_uint64)]),
+    "seg_launch_count": (c_int32, [c_void_p, POINTER(c_uint64)]),
+    "seg_poll_status": (c_int32, [c_void_p]),
+    "seg_timer_start": (c_int32, [c_void_p]),
+    "seg_timer_stop": (c_int32, [c_void_p]),
+    "seg_timer_elapsed_ms": (c_int32, [c_void_p, POINTER(c_float)]),
+    "seg_profile_enable": (c_int32, [c_void_p, c_int32]),
+    "seg_profile_get": (c_int32, [c_void_p, c_int32, POINTER(c_uint64), POINTER(c_float)]),
+    "seg_status_string": (c_char_p, [c_int32]),
+    "seg_last_error": (c_char_p, [c_void_p]),
+    "seg_build_info": (c_char_p, []),
+}
+
+_lib = None
+
+
+def load():
+    """Loads the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2403_11204_b200.build` "
+                               "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+class SegError(RuntimeError):
+    def __init__(self, status, detail=""):
+        self.status = status
+        msg = load().seg_status_string(status).decode()
+        super().__init__(f"seg status {status}: {msg}" + (f" ({detail})" if detail else ""))
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+class Segment:
+    """One network segment on the current CUDA device.  Tensors are torch CUDA tensors."""
+
+    def __init__(self, widths, n_classes, is_final, *, precision="fp32", optimizer="sgd", lr=0.01,
+                 momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, max_batch=256, segment_id=0,
+                 init_seed=2, last_relu=None, gemm_backend="auto", stream=None):
+        import torch
+        self._torch = torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("Segment needs a CUDA device; there is no CPU path")
+        self.lib = load()
+        self.widths = [int(w) for w in widths]
+        self.n_layers = len(self.widths) - 1
+        self.n_classes, self.is_final, self.precision = int(n_classes), bool(is_final), precision
+        self.max_batch = int(max_batch)
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self._warr = (c_int32 * len(self.widths))(*self.widths)
+        cfg = seg_config(self.n_layers, self._warr, self.n_classes, int(self.is_final),
+                         -1 if last_relu is None else int(bool(last_relu)), int(segment_id),
+                         PRECISIONS[precision], OPTIMIZERS[optimizer], lr, momentum, beta1, beta2, eps,
+                         self.max_batch, BACKENDS[gemm_backend], int(init_seed),
+                         c_void_p(self.stream.cuda_stream))
+        self.h = c_void_p()
+        self._check(self.lib.seg_create(byref(cfg), byref(self.h)), "seg_create")
+        self.act_dtype = torch.bfloat16 if precision == "bf16" else torch.float32
+        self.out_dtype = torch.float32 if self.is_final else self.act_dtype
+        self.last_batch = 0
+
+    # -- plumbing -------------------------------------------------------------------------
+    def _check(self, status, what=""):
+        if status != SEG_OK:
+            detail = what
+            if self.h:
+                err = self.lib.seg_last_error(self.h).decode()
+                detail = f"{what}: {err}" if err else what
+            raise SegError(status, detail)
+
+    def _empty(self, *shape, dtype=None):
+        with self._torch.cuda.stream(self.stream):
+            return self._torch.empty(*shape, dtype=dtype or self._torch.float32, device="cuda")
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.seg_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the five calls -------------------------------------------------------------------------
+    def gen_labels(self, seed, dist="uniform_kappa", kappa=10.0):
+        self._check(self.lib.seg_gen_labels(self.h, int(seed), LABEL_DISTS[dist], float(kappa)), "seg_gen_labels")
+
+    def train_step(self, x, cls, loss_out=None, y_out=None):
+        batch = x.shape[0]
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.act_dtype and x.shape[1] == self.widths[0]
+        assert cls.is_cuda and cls.is_contiguous() and cls.dtype == self._torch.int32 and cls.shape[0] == batch
+        self._check(self.lib.seg_train_step(self.h, _ptr(x), _ptr(cls), batch, _ptr(loss_out), _ptr(y_out)),
+                    "seg_train_step")
+        self.last_batch = batch
+
+    def train_step_host(self, x_host, cls_host):
+        """x_host / cls_host: CPU tensors (pinned for speed).  Returns the loss as a float."""
+        batch = x_host.shape[0]
+        assert not x_host.is_cuda and x_host.is_contiguous() and x_host.dtype == self.act_dtype
+        assert not cls_host.is_cuda and cls_host.dtype == self._torch.int32
+        loss = c_float()
+        self._check(self.lib.seg_train_step_host(self.h, c_void_p(x_host.data_ptr()),
+                                                 c_void_p(cls_host.data_ptr()), batch, byref(loss)),
+                    "seg_train_step_host")
+        self.last_batch = batch
+        return loss.value
+
+    def forward(self, x, y=None):
+        batch = x.shape[0]
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.act_dtype and x.shape[1] == self.widths[0]
+        if y is None:
+            y = self._empty(batch, self.widths[-1], dtype=self.out_dtype)
+        self._check(self.lib.seg_forward(self.h, _ptr(x), batch, _ptr(y)), "seg_forward")
+        self.last_batch = batch
+        return y
+
+    # -- inspection -------------------------------------------------------------------------
+    def labels(self):
+        t = self._empty(self.n_classes, self.widths[-1])
+        self._check(self.lib.seg_get_labels(self.h, _ptr(t)), "seg_get_labels")
+        return t
+
+    def set_labels(self, t):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == self._torch.float32
+        self._check(self.lib.seg_set_labels(self.h, _ptr(t)), "seg_set_labels")
+
+    def _pair(self, fn, layer, *extra):
+        w = self._empty(self.widths[layer + 1], self.widths[layer])
+        b = self._empty(self.widths[layer + 1])
+        self._check(fn(self.h, layer, *extra, _ptr(w), _ptr(b)), fn.__name__)
+        return w, b
+
+    def params(self, layer):
+        return self._pair(self.lib.seg_get_params, layer)
+
+    def grads(self, layer):
+        return self._pair(self.lib.seg_get_grads, layer)
+
+    def opt_state(self, layer, which):
+        return self._pair(self.lib.seg_get_opt_state, layer, which)
+
+    def set_params(self, layer, W, b):
+        W = W.contiguous().float()
+        b = b.contiguous().float()
+        self._check(self.lib.seg_set_params(self.h, layer, _ptr(W), _ptr(b)), "seg_set_params")
+        self.stream.synchronize()
+
+    def activation(self, layer):
+        t = self._empty(self.last_batch, self.widths[layer])
+        self._check(self.lib.seg_get_activation(self.h, layer, _ptr(t)), "seg_get_activation")
+        return t
+
+    def mem_bytes(self):
+        cur, peak = c_uint64(), c_uint64()
+        self._check(self.lib.seg_mem_bytes(self.h, byref(cur), byref(peak)), "seg_mem_bytes")
+        return cur.value, peak.value
+
+    def launch_count(self):
+        n = c_uint64()
+        self._check(self.lib.seg_launch_count(self.h, byref(n)), "seg_launch_count")
+        return n.value
+
+    def poll(self):
+        self._check(self.lib.seg_poll_status(self.h), "seg_poll_status")
+
+    def timer_start(self):
+        self._check(self.lib.seg_timer_start(self.h))
+
+    def timer_stop(self):
+        self._check(self.lib.seg_timer_stop(self.h))
+
+    def timer_ms(self):
+        ms = c_float()
+        self._check(self.lib.seg_timer_elapsed_ms(self.h, byref(ms)))
+        return ms.value
+
+    def profile(self, on):
+        self._check(self.lib.seg_profile_enable(self.h, int(on)))
+
+    def profile_read(self):
+        out = {}
+        for k, name in enumerate(KERNEL_KINDS):
+            n, ms = c_uint64(), c_float()
+            self._check(self.lib.seg_profile_get(self.h, k, byref(n), byref(ms)))
+            out[name] = (n.value, ms.value)
+        return out

@@ -1,0 +1,110 @@
+// Shared declarations of the segment-trainer library (internal; the public ABI is include/seg.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "seg.h"
+
+namespace segk {
+
+// Storage type of an operand / activation buffer.
+enum DType : int { DT_F32 = 0, DT_BF16 = 1 };
+// Rounding applied when a value is stored into a buffer that later feeds a matrix product.
+enum Round : int { RND_NONE = 0, RND_TF32 = 1, RND_BF16 = 2 };
+
+// Epilogues of the three matrix products of a Linear layer.
+enum Epilogue : int {
+  EPI_BIAS_ACT = 0,  // forward: + bias[n], optional ReLU
+  EPI_MASK = 1,      // dgrad:   * (mask[m][n] > 0)  (mask = stored post-ReLU activation)
+  EPI_PLAIN = 2      // wgrad:   store the fp32 product
+};
+
+// Device status word values (written by kernels that give up a bounded wait).
+enum DevStatus : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
+
+// One matrix product  C[M][N] = sum_k A(m,k) * B(k,n)  with explicit element strides, so that
+// forward (A W^T), dgrad (dZ W) and wgrad (dZ^T A) are all expressed by one description.
+struct GemmDesc {
+  const void* A;   // element (m,k) at A + m*a_sm + k*a_sk   (elements of a_dt)
+  const void* B;   // element (k,n) at B + k*b_sk + n*b_sn   (elements of b_dt)
+  void* C;         // element (m,n) at C + m*ldc + n         (elements of c_dt)
+  int64_t a_sm, a_sk, b_sk, b_sn, ldc;
+  int M, N, K;
+  int a_dt, b_dt, c_dt;     // DType
+  int c_round;              // Round applied to C on store
+  int epi;                  // Epilogue
+  int relu;                 // EPI_BIAS_ACT: apply ReLU
+  const float* bias;        // EPI_BIAS_ACT: [N]
+  const void* mask;         // EPI_MASK: [M][ldmask] of c_dt
+  int64_t ldmask;
+};
+
+// ---- launchers (each returns the cudaError_t of its launch) -------------------------------
+cudaError_t launch_gemm_simt(const GemmDesc& g, cudaStream_t s);
+// Tensor-core path.  Returns cudaErrorNotSupported when the shape/stride does not fit its TMA rules.
+cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s);
+bool gemm_tc_init();   // resolves the driver entry point needed for tensor maps
+
+cudaError_t launch_gen_labels(float* dst, int n_classes, int n_p, uint64_t seed, int segment_id,
+                              int dist, float kappa, cudaStream_t s);
+cudaError_t launch_init_uniform(float* dst, int rows, int cols, int64_t ld, uint64_t seed,
+                                int segment_id, int layer, int tag, float bound, cudaStream_t s);
+
+// loss kernels: write dZ (dz_dt, rounded by dz_round) and a deterministic batch loss
+cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const int32_t* cls,
+                            const float* sil, int n_p, int batch, int relu_mask,
+                            void* dz, int dz_dt, int dz_round, int64_t ld_dz,
+                            float* partials, unsigned int* counter, float* loss_out, cudaStream_t s);
+cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const int32_t* cls,
+                                   int n_classes, int batch, int relu_mask,
+                                   void* dz, int dz_dt, int dz_round, int64_t ld_dz,
+                                   float* partials, unsigned int* counter, float* loss_out,
+                                   cudaStream_t s);
+int loss_max_partials();
+
+// db[n] = sum_b dZ[b][n], deterministic
+cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, int n, float* db,
+                             float* scratch, cudaStream_t s);
+int bias_grad_scratch_floats(int batch, int n);
+
+struct UpdateArgs {
+  float* p; const float* g; float* s1; float* s2;
+  void* p_op;          // reduced-precision operand copy (may be null)
+  int op_dt;           // DType of p_op
+  int op_round;        // Round for p_op
+  int64_t n;
+  int optimizer;
+  float lr, momentum, beta1, beta2, eps;
+  float bc1, bc2;      // Adam bias corrections 1-b1^t, 1-b2^t
+};
+cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s);
+
+// copies with pitch / dtype / rounding conversion: dst[r][c] = cvt(src[r][c])
+cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt,
+                          int64_t ld_src, int rows, int cols, int round, cudaStream_t s);
+
+// ---- small device helpers ------------------------------------------------------------------
+__device__ __forceinline__ float round_tf32_rne(float x) {
+  uint32_t u = __float_as_uint(x);
+  u = (u + 0x0FFFu + ((u >> 13) & 1u)) & 0xFFFFE000u;
+  return __uint_as_float(u);
+}
+__device__ __forceinline__ float round_bf16_rne(float x) {
+  return __bfloat162float(__float2bfloat16_rn(x));
+}
+__device__ __forceinline__ float apply_round(float x, int mode) {
+  if (mode == RND_TF32) return round_tf32_rne(x);
+  if (mode == RND_BF16) return round_bf16_rne(x);
+  return x;
+}
+__device__ __forceinline__ float load_as_float(const void* p, int dt, int64_t i) {
+  return dt == DT_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
+                       : reinterpret_cast<const float*>(p)[i];
+}
+__device__ __forceinline__ void store_from_float(void* p, int dt, int64_t i, float v) {
+  if (dt == DT_BF16) reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(p)[i] = v;
+}
+
+}  // namespace segk

@@ -1,0 +1,316 @@
+// Streaming kernels of the segment step: the two losses (Section 2: intermediate-label
+// regression for a non-final segment, class labels for the final one), the bias gradient,
+// the fused optimizer update (Section 3: SGD with momentum; plain SGD and Adam as well) and
+// pitch/dtype conversion copies.  All of them are HBM-bound; none uses tensor cores.
+#include "common.cuh"
+
+namespace segk {
+namespace {
+
+constexpr int kLossThreads = 256;
+constexpr int kMaxLossBlocks = 1024;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+
+// Sum over the block in a fixed order (deterministic for a fixed launch shape).
+__device__ float block_sum(float v, float* smem /* >= 32 floats */) {
+  v = warp_sum(v);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane == 0) smem[warp] = v;
+  __syncthreads();
+  float total = 0.f;
+  if (warp == 0) {
+    const int n_warps = (blockDim.x + 31) >> 5;
+    total = lane < n_warps ? smem[lane] : 0.f;
+    total = warp_sum(total);
+  }
+  return total;  // valid in warp 0
+}
+
+// Writes this block's partial; the last block to finish adds all partials in index order and
+// writes loss_out = scale * total.  The counter is left at zero for the next launch.
+__device__ void finish_loss(float block_total, float* partials, unsigned int* counter,
+                            float* loss_out, float scale, float* smem) {
+  __shared__ bool is_last;
+  if (threadIdx.x == 0) {
+    partials[blockIdx.x] = block_total;
+    __threadfence();
+    const unsigned int done = atomicAdd(counter, 1u);
+    is_last = (done == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    float v = 0.f;
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += blockDim.x) v += __ldcg(partials + i);
+    const float total = block_sum(v, smem);
+    if (threadIdx.x == 0) {
+      if (loss_out) *loss_out = total * scale;
+      *counter = 0u;
+    }
+  }
+}
+
+// Non-final segment: target of sample b is row cls[b] of the label matrix (gathered here, never
+// materialised per sample);  loss = mean (a - t)^2,  dZ = 2 (a - t) / (B N_P) * [a > 0].
+template <typename TOut, typename TDz>
+__global__ void __launch_bounds__(kLossThreads)
+mse_loss_kernel(const TOut* __restrict__ out, int64_t ld_out, const int32_t* __restrict__ cls,
+                const float* __restrict__ sil, int n_p, int batch, int relu_mask,
+                TDz* __restrict__ dz, int dz_round, int64_t ld_dz, float* partials,
+                unsigned int* counter, float* loss_out) {
+  __shared__ float red[32];
+  const int64_t total = (int64_t)batch * n_p;
+  const float gscale = 2.0f / (float)total;
+  float acc = 0.f;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
+       e += (int64_t)gridDim.x * blockDim.x) {
+    const int b = (int)(e / n_p), i = (int)(e % n_p);
+    float a;
+    if constexpr (sizeof(TOut) == 2) a = __bfloat162float(out[b * ld_out + i]);
+    else a = out[b * ld_out + i];
+    const float t = __ldg(sil + (int64_t)__ldg(cls + b) * n_p + i);
+    const float d = a - t;
+    acc = fmaf(d, d, acc);
+    float g = d * gscale;
+    if (relu_mask && !(a > 0.f)) g = 0.f;
+    g = apply_round(g, dz_round);
+    if constexpr (sizeof(TDz) == 2) dz[b * ld_dz + i] = __float2bfloat16_rn(g);
+    else dz[b * ld_dz + i] = g;
+  }
+  const float bt = block_sum(acc, red);
+  finish_loss(bt, partials, counter, loss_out, 1.0f / (float)total, red);
+}
+
+// Final segment: one warp per sample;  p = softmax(z) with the row maximum subtracted,
+// loss = -mean log p[cls],  dZ = (p - onehot) / B.
+template <typename TDz>
+__global__ void __launch_bounds__(kLossThreads)
+softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* __restrict__ cls,
+                  int n_classes, int batch, int relu_mask, TDz* __restrict__ dz, int dz_round,
+                  int64_t ld_dz, float* partials, unsigned int* counter, float* loss_out) {
+  __shared__ float red[32];
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  const float inv_b = 1.0f / (float)batch;
+  float acc = 0.f;
+  for (int b = blockIdx.x * warps_per_block + (threadIdx.x >> 5); b < batch;
+       b += gridDim.x * warps_per_block) {
+    const float* z = logits + (int64_t)b * ld;
+    float mx = -INFINITY;
+    for (int i = lane; i < n_classes; i += 32) mx = fmaxf(mx, z[i]);
+    mx = warp_max(mx);
+    float se = 0.f;
+    for (int i = lane; i < n_classes; i += 32) se += expf(z[i] - mx);
+    se = warp_sum(se);
+    const int c = __ldg(cls + b);
+    const float inv_se = 1.0f / se;
+    for (int i = lane; i < n_classes; i += 32) {
+      const float zi = z[i];
+      float g = (expf(zi - mx) * inv_se - (i == c ? 1.f : 0.f)) * inv_b;
+      if (relu_mask && !(zi > 0.f)) g = 0.f;
+      g = apply_round(g, dz_round);
+      if constexpr (sizeof(TDz) == 2) dz[(int64_t)b * ld_dz + i] = __float2bfloat16_rn(g);
+      else dz[(int64_t)b * ld_dz + i] = g;
+    }
+    if (lane == 0) acc += logf(se) - (z[c] - mx);
+  }
+  const float bt = block_sum(acc, red);
+  finish_loss(bt, partials, counter, loss_out, inv_b, red);
+}
+
+// db[n] = sum_b dZ[b][n]: 32 columns x 8 row lanes per block, fixed summation order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bias_grad_kernel(const T* __restrict__ dz, int64_t ld, int batch, int n, float* __restrict__ db) {
+  __shared__ float part[8][33];
+  const int col = blockIdx.x * 32 + (threadIdx.x & 31);
+  const int rl = threadIdx.x >> 5;
+  float acc = 0.f;
+  if (col < n) {
+#pragma unroll 4
+    for (int b = rl; b < batch; b += 8) {
+      if constexpr (sizeof(T) == 2) acc += __bfloat162float(dz[(int64_t)b * ld + col]);
+      else acc += dz[(int64_t)b * ld + col];
+    }
+  }
+  part[rl][threadIdx.x & 31] = acc;
+  __syncthreads();
+  if (rl == 0 && col < n) {
+    float s = 0.f;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) s += part[r][threadIdx.x & 31];
+    db[col] = s;
+  }
+}
+
+// One pass over the flat parameter range of a segment: parameters, gradients and optimizer
+// state share one layout, so a single launch updates every tensor and refreshes the
+// reduced-precision operand copy.
+template <int OPT, int OPDT>
+__global__ void __launch_bounds__(256)
+update_kernel(UpdateArgs u) {
+  const int64_t n4 = u.n >> 2;
+  float4* __restrict__ p4 = reinterpret_cast<float4*>(u.p);
+  const float4* __restrict__ g4 = reinterpret_cast<const float4*>(u.g);
+  float4* __restrict__ s14 = reinterpret_cast<float4*>(u.s1);
+  float4* __restrict__ s24 = reinterpret_cast<float4*>(u.s2);
+  const float inv_bc1 = 1.0f / u.bc1, inv_bc2 = 1.0f / u.bc2;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    float4 p = p4[i];
+    const float4 g = g4[i];
+    float pv[4] = {p.x, p.y, p.z, p.w};
+    const float gv[4] = {g.x, g.y, g.z, g.w};
+    if constexpr (OPT == SEG_SGD) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) pv[k] = pv[k] - u.lr * gv[k];
+    } else if constexpr (OPT == SEG_SGD_MOMENTUM) {
+      float4 m = s14[i];
+      float mv[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        mv[k] = u.momentum * mv[k] + gv[k];
+        pv[k] = pv[k] - u.lr * mv[k];
+      }
+      s14[i] = make_float4(mv[0], mv[1], mv[2], mv[3]);
+    } else {
+      float4 m = s14[i], v = s24[i];
+      float mv[4] = {m.x, m.y, m.z, m.w}, vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        mv[k] = u.beta1 * mv[k] + (1.0f - u.beta1) * gv[k];
+        vv[k] = u.beta2 * vv[k] + (1.0f - u.beta2) * gv[k] * gv[k];
+        const float mhat = mv[k] * inv_bc1;
+        const float vhat = vv[k] * inv_bc2;
+        pv[k] = pv[k] - u.lr * mhat / (sqrtf(vhat) + u.eps);
+      }
+      s14[i] = make_float4(mv[0], mv[1], mv[2], mv[3]);
+      s24[i] = make_float4(vv[0], vv[1], vv[2], vv[3]);
+    }
+    p4[i] = make_float4(pv[0], pv[1], pv[2], pv[3]);
+    if constexpr (OPDT == DT_BF16) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(pv[0], pv[1]);
+      __nv_bfloat162 hi = __floats2bfloat162_rn(pv[2], pv[3]);
+      uint2 packed;
+      packed.x = *reinterpret_cast<uint32_t*>(&lo);
+      packed.y = *reinterpret_cast<uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(u.p_op)[i] = packed;
+    } else if constexpr (OPDT == DT_F32) {
+      if (u.p_op != nullptr) {
+        reinterpret_cast<float4*>(u.p_op)[i] =
+            make_float4(apply_round(pv[0], u.op_round), apply_round(pv[1], u.op_round),
+                        apply_round(pv[2], u.op_round), apply_round(pv[3], u.op_round));
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt, int64_t ld_src,
+              int rows, int cols, int round) {
+  const int64_t total = (int64_t)rows * cols;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
+       e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = e / cols, c = e % cols;
+    const float v = apply_round(load_as_float(src, src_dt, r * ld_src + c), round);
+    store_from_float(dst, dst_dt, r * ld_dst + c, v);
+  }
+}
+
+int grid_for(int64_t work_items, int threads, int max_blocks) {
+  int64_t b = (work_items + threads - 1) / threads;
+  if (b < 1) b = 1;
+  return (int)(b < max_blocks ? b : max_blocks);
+}
+
+}  // namespace
+
+int loss_max_partials() { return kMaxLossBlocks; }
+
+cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const int32_t* cls,
+                            const float* sil, int n_p, int batch, int relu_mask, void* dz,
+                            int dz_dt, int dz_round, int64_t ld_dz, float* partials,
+                            unsigned int* counter, float* loss_out, cudaStream_t s) {
+  const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
+  if (out_dt == DT_BF16 && dz_dt == DT_BF16) {
+    mse_loss_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, kLossThreads, 0, s>>>(
+        (const __nv_bfloat16*)out, ld_out, cls, sil, n_p, batch, relu_mask, (__nv_bfloat16*)dz,
+        dz_round, ld_dz, partials, counter, loss_out);
+  } else if (out_dt == DT_F32 && dz_dt == DT_F32) {
+    mse_loss_kernel<float, float><<<grid, kLossThreads, 0, s>>>(
+        (const float*)out, ld_out, cls, sil, n_p, batch, relu_mask, (float*)dz, dz_round, ld_dz,
+        partials, counter, loss_out);
+  } else {
+    return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const int32_t* cls,
+                                   int n_classes, int batch, int relu_mask, void* dz, int dz_dt,
+                                   int dz_round, int64_t ld_dz, float* partials,
+                                   unsigned int* counter, float* loss_out, cudaStream_t s) {
+  const int warps = kLossThreads / 32;
+  const int grid = grid_for(batch, warps, kMaxLossBlocks);
+  if (dz_dt == DT_BF16) {
+    softmax_ce_kernel<__nv_bfloat16><<<grid, kLossThreads, 0, s>>>(
+        logits, ld_logits, cls, n_classes, batch, relu_mask, (__nv_bfloat16*)dz, dz_round, ld_dz,
+        partials, counter, loss_out);
+  } else {
+    softmax_ce_kernel<float><<<grid, kLossThreads, 0, s>>>(logits, ld_logits, cls, n_classes,
+                                                          batch, relu_mask, (float*)dz, dz_round,
+                                                          ld_dz, partials, counter, loss_out);
+  }
+  return cudaGetLastError();
+}
+
+int bias_grad_scratch_floats(int, int) { return 0; }
+
+cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, int n, float* db,
+                             float*, cudaStream_t s) {
+  const int grid = (n + 31) / 32;
+  if (dz_dt == DT_BF16)
+    bias_grad_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)dz, ld, batch, n, db);
+  else
+    bias_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dz, ld, batch, n, db);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
+  if (u.n == 0) return cudaSuccess;
+  if (u.n & 3) return cudaErrorInvalidValue;
+  const int grid = grid_for(u.n >> 2, 256, 148 * 8);
+  const bool bf = (u.p_op != nullptr && u.op_dt == DT_BF16);
+#define SEGK_UPD(OPT)                                                      \
+  if (bf) update_kernel<OPT, DT_BF16><<<grid, 256, 0, s>>>(u);             \
+  else update_kernel<OPT, DT_F32><<<grid, 256, 0, s>>>(u)
+  switch (u.optimizer) {
+    case SEG_SGD: SEGK_UPD(SEG_SGD); break;
+    case SEG_SGD_MOMENTUM: SEGK_UPD(SEG_SGD_MOMENTUM); break;
+    case SEG_ADAM: SEGK_UPD(SEG_ADAM); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef SEGK_UPD
+  return cudaGetLastError();
+}
+
+cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt,
+                          int64_t ld_src, int rows, int cols, int round, cudaStream_t s) {
+  if ((int64_t)rows * cols == 0) return cudaSuccess;
+  const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
+  copy2d_kernel<<<grid, 256, 0, s>>>(dst, dst_dt, ld_dst, src, src_dt, ld_src, rows, cols, round);
+  return cudaGetLastError();
+}
+
+}  // namespace segk

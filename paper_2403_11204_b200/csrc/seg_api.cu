@@ -1,0 +1,600 @@
+// C ABI of the segment trainer (declared in include/seg.h): handle, workspace layout, and the
+// order in which one training step enqueues its kernels.
+//
+// Device memory layout of a handle
+//   params / grads / state1 / state2 : one flat fp32 range each, identical layout
+//       [W_0 | b_0 | W_1 | b_1 | ...], every tensor starting on a 256-byte boundary, W_l stored
+//       [out][ldw] with ldw = in rounded up to 8 elements (16-byte rows for TMA); padding stays 0.
+//   params_op : the same layout in the operand dtype (bf16, or TF32-rounded fp32).
+//   act[l], l = 1..L : [max_batch][ld_l] stored outputs (bf16 or fp32; final logits fp32).
+//   dz[0], dz[1]     : ping-pong dZ buffers, [max_batch][max ld].
+//   sil              : [M][N_P] fp32 intermediate labels (Eq. 1).
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace segk;
+
+namespace {
+
+struct LayerInfo {
+  int in, out;
+  int64_t ldw;
+  int64_t w_off, b_off;  // element offsets into the flat ranges
+};
+
+enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_BIAS, K_UPDATE, K_COPY, K_COUNT };
+
+int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+struct seg_handle {
+  int n_layers = 0, n_classes = 0, max_batch = 0, segment_id = 0;
+  bool is_final = false, last_relu = false;
+  int precision = SEG_FP32, optimizer = SEG_SGD;
+  float lr = 0, momentum = 0, beta1 = 0, beta2 = 0, eps = 0;
+  uint64_t init_seed = 0;
+  cudaStream_t stream = nullptr;
+  bool use_tc = false;
+  int act_dt = DT_F32, act_round = RND_NONE, op_dt = DT_F32, op_round = RND_NONE;
+  std::vector<int> widths;
+  std::vector<LayerInfo> layers;
+  int64_t n_flat = 0;
+  float *params = nullptr, *grads = nullptr, *state1 = nullptr, *state2 = nullptr;
+  void* params_op = nullptr;
+  std::vector<void*> act;          // index 1..L
+  std::vector<int64_t> ld_act;     // index 0..L
+  std::vector<int> act_dtype;      // index 1..L
+  void* x_stage = nullptr;
+  void* dz[2] = {nullptr, nullptr};
+  float* sil = nullptr;
+  bool have_labels = false;
+  float* loss_partials = nullptr;
+  unsigned int* loss_counter = nullptr;
+  int* dev_status = nullptr;
+  void* host_x = nullptr;          // device staging of seg_train_step_host
+  int32_t* host_cls = nullptr;
+  float* host_loss = nullptr;
+  int last_batch = 0;
+  uint64_t step = 0;
+  uint64_t mem_current = 0, mem_peak = 0, launches = 0;
+  std::vector<void*> allocations;
+  cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  bool profile = false;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  std::vector<int> ev_kind;        // kind of each recorded pair
+  std::string last_error;
+};
+
+namespace {
+
+seg_status fail_cuda(seg_handle* h, cudaError_t e, const char* what) {
+  if (h) h->last_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return e == cudaErrorMemoryAllocation ? SEG_ERR_ALLOC : SEG_ERR_CUDA;
+}
+
+#define SEG_TRY(h, expr, what)                                   \
+  do {                                                           \
+    cudaError_t e__ = (expr);                                    \
+    if (e__ != cudaSuccess) return fail_cuda((h), e__, (what));  \
+  } while (0)
+
+template <typename T>
+seg_status dev_alloc(seg_handle* h, T** out, size_t count, bool zero) {
+  const size_t bytes = round_up((int64_t)(count * sizeof(T)), 256);
+  void* p = nullptr;
+  if (bytes == 0) { *out = nullptr; return SEG_OK; }
+  cudaError_t e = cudaMalloc(&p, bytes);
+  if (e != cudaSuccess) { cudaGetLastError(); return fail_cuda(h, e, "cudaMalloc"); }
+  h->allocations.push_back(p);
+  h->mem_current += bytes;
+  if (h->mem_current > h->mem_peak) h->mem_peak = h->mem_current;
+  if (zero) SEG_TRY(h, cudaMemsetAsync(p, 0, bytes, h->stream), "cudaMemsetAsync");
+  *out = reinterpret_cast<T*>(p);
+  return SEG_OK;
+}
+
+// Brackets one launch with events while profiling is on.
+struct Launch {
+  seg_handle* h;
+  bool on;
+  Launch(seg_handle* hh, int kind) : h(hh), on(hh->profile) {
+    ++h->launches;
+    if (!on) return;
+    if (h->ev_used + 2 > h->ev_pool.size()) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+        h->ev_pool.push_back(e);
+      }
+    }
+    cudaEventRecord(h->ev_pool[h->ev_used], h->stream);
+    h->ev_kind.push_back(kind);
+  }
+  ~Launch() {
+    if (!on) return;
+    cudaEventRecord(h->ev_pool[h->ev_used + 1], h->stream);
+    h->ev_used += 2;
+  }
+};
+
+seg_status run_gemm(seg_handle* h, const GemmDesc& g, int kind) {
+  Launch l(h, kind);
+  if (h->use_tc) {
+    cudaError_t e = launch_gemm_tc(g, h->dev_status, h->stream);
+    if (e == cudaSuccess) return SEG_OK;
+    if (e != cudaErrorNotSupported) return fail_cuda(h, e, "tensor-core product launch");
+    cudaGetLastError();
+  }
+  SEG_TRY(h, launch_gemm_simt(g, h->stream), "FFMA product launch");
+  return SEG_OK;
+}
+
+size_t elem_size(int dt) { return dt == DT_BF16 ? 2 : 4; }
+
+void* weights_op(seg_handle* h, int l) {
+  char* base = reinterpret_cast<char*>(h->params_op ? h->params_op : (void*)h->params);
+  return base + h->layers[l].w_off * elem_size(h->params_op ? h->op_dt : DT_F32);
+}
+
+// Returns the pointer / pitch the first product reads x from, staging it when the caller's
+// buffer cannot be used directly (TF32 rounding, or rows that are not 16-byte multiples).
+seg_status prepare_input(seg_handle* h, const void* x, int batch, const void** x_use, int64_t* ld) {
+  const int w0 = h->widths[0];
+  const bool aligned = ((reinterpret_cast<uintptr_t>(x) & 15u) == 0) &&
+                       ((w0 * elem_size(h->act_dt)) % 16 == 0);
+  if (h->precision != SEG_TF32 && (aligned || !h->use_tc)) {
+    *x_use = x; *ld = w0;
+    return SEG_OK;
+  }
+  Launch l(h, K_COPY);
+  SEG_TRY(h, launch_copy2d(h->x_stage, h->act_dt, h->ld_act[0], x, h->act_dt, w0, batch, w0,
+                           h->act_round, h->stream), "input staging");
+  *x_use = h->x_stage; *ld = h->ld_act[0];
+  return SEG_OK;
+}
+
+seg_status forward_impl(seg_handle* h, const void* x, int batch, const void** x_use, int64_t* ld_x) {
+  const void* a_prev; int64_t ld_prev;
+  seg_status st = prepare_input(h, x, batch, &a_prev, &ld_prev);
+  if (st != SEG_OK) return st;
+  *x_use = a_prev; *ld_x = ld_prev;
+  for (int l = 0; l < h->n_layers; ++l) {
+    const LayerInfo& L = h->layers[l];
+    const bool last = (l == h->n_layers - 1);
+    GemmDesc g{};
+    g.A = a_prev; g.a_sm = ld_prev; g.a_sk = 1; g.a_dt = h->act_dt;
+    g.B = weights_op(h, l); g.b_sk = 1; g.b_sn = L.ldw; g.b_dt = h->op_dt;
+    g.C = h->act[l + 1]; g.ldc = h->ld_act[l + 1]; g.c_dt = h->act_dtype[l + 1];
+    g.M = batch; g.N = L.out; g.K = L.in;
+    g.c_round = (last && h->is_final) ? RND_NONE : h->act_round;
+    g.epi = EPI_BIAS_ACT; g.relu = (!last || h->last_relu) ? 1 : 0;
+    g.bias = h->params + L.b_off;
+    st = run_gemm(h, g, K_FWD);
+    if (st != SEG_OK) return st;
+    a_prev = h->act[l + 1]; ld_prev = h->ld_act[l + 1];
+  }
+  h->last_batch = batch;
+  return SEG_OK;
+}
+
+seg_status copy_out(seg_handle* h, void* y, int batch) {
+  const int L = h->n_layers;
+  Launch l(h, K_COPY);
+  SEG_TRY(h, launch_copy2d(y, h->act_dtype[L], h->widths[L], h->act[L], h->act_dtype[L],
+                           h->ld_act[L], batch, h->widths[L], RND_NONE, h->stream), "output copy");
+  return SEG_OK;
+}
+
+seg_status refresh_operand_copy(seg_handle* h, int64_t off, int64_t n) {
+  if (!h->params_op || n == 0) return SEG_OK;
+  Launch l(h, K_COPY);
+  char* dst = reinterpret_cast<char*>(h->params_op) + off * elem_size(h->op_dt);
+  SEG_TRY(h, launch_copy2d(dst, h->op_dt, n, h->params + off, DT_F32, n, 1, (int)n, h->op_round,
+                           h->stream), "operand copy refresh");
+  return SEG_OK;
+}
+
+bool valid_layer(const seg_handle* h, int layer) { return layer >= 0 && layer < h->n_layers; }
+
+}  // namespace
+
+extern "C" {
+
+const char* seg_status_string(int32_t s) {
+  switch (s) {
+    case SEG_OK: return "ok";
+    case SEG_ERR_INVALID_ARG: return "invalid argument";
+    case SEG_ERR_SHAPE: return "shape out of range";
+    case SEG_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SEG_ERR_ALLOC: return "device allocation failed";
+    case SEG_ERR_CUDA: return "CUDA call failed";
+    case SEG_ERR_STATE: return "call not valid in this state";
+    case SEG_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait";
+    case SEG_ERR_NO_DEVICE: return "no usable CUDA device";
+    default: return "unknown status";
+  }
+}
+
+const char* seg_build_info(void) { return "segment trainer for sm_100a (tcgen05/TMEM/TMA products, FFMA fp32 path)"; }
+
+const char* seg_last_error(const seg_handle* h) { return h ? h->last_error.c_str() : ""; }
+
+seg_status seg_create(const seg_config* cfg, seg_handle** out) {
+  if (!out) return SEG_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg || !cfg->widths) return SEG_ERR_INVALID_ARG;
+  if (cfg->n_layers < 1 || cfg->n_layers > 16) return SEG_ERR_SHAPE;
+  if (cfg->n_classes < 1 || cfg->max_batch < 1) return SEG_ERR_SHAPE;
+  for (int i = 0; i <= cfg->n_layers; ++i)
+    if (cfg->widths[i] < 1 || cfg->widths[i] > (1 << 20)) return SEG_ERR_SHAPE;
+  if (cfg->precision < SEG_FP32 || cfg->precision > SEG_BF16) return SEG_ERR_INVALID_ARG;
+  if (cfg->optimizer < SEG_SGD || cfg->optimizer > SEG_ADAM) return SEG_ERR_INVALID_ARG;
+  if (cfg->gemm_backend < SEG_GEMM_AUTO || cfg->gemm_backend > SEG_GEMM_TCGEN05) return SEG_ERR_INVALID_ARG;
+  if (cfg->gemm_backend == SEG_GEMM_TCGEN05 && cfg->precision == SEG_FP32) return SEG_ERR_UNSUPPORTED;
+  if (cfg->is_final && cfg->widths[cfg->n_layers] != cfg->n_classes) return SEG_ERR_SHAPE;
+  if (!(cfg->lr >= 0.f)) return SEG_ERR_INVALID_ARG;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SEG_ERR_NO_DEVICE; }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { cudaGetLastError(); return SEG_ERR_NO_DEVICE; }
+  if (prop.major != 10) return SEG_ERR_NO_DEVICE;
+
+  seg_handle* h = new (std::nothrow) seg_handle();
+  if (!h) return SEG_ERR_ALLOC;
+  h->n_layers = cfg->n_layers; h->n_classes = cfg->n_classes; h->max_batch = cfg->max_batch;
+  h->segment_id = cfg->segment_id; h->is_final = cfg->is_final != 0;
+  h->last_relu = cfg->last_relu < 0 ? !h->is_final : (cfg->last_relu != 0);
+  h->precision = cfg->precision; h->optimizer = cfg->optimizer;
+  h->lr = cfg->lr; h->momentum = cfg->momentum; h->beta1 = cfg->beta1; h->beta2 = cfg->beta2;
+  h->eps = cfg->eps; h->init_seed = cfg->init_seed;
+  h->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
+  h->widths.assign(cfg->widths, cfg->widths + cfg->n_layers + 1);
+  if (h->precision == SEG_BF16) { h->act_dt = DT_BF16; h->act_round = RND_BF16; h->op_dt = DT_BF16; h->op_round = RND_BF16; }
+  if (h->precision == SEG_TF32) { h->act_round = RND_TF32; h->op_round = RND_TF32; }
+  h->use_tc = (h->precision != SEG_FP32) && (cfg->gemm_backend != SEG_GEMM_SIMT);
+  if (h->use_tc && !gemm_tc_init()) {
+    if (cfg->gemm_backend == SEG_GEMM_TCGEN05) { delete h; return SEG_ERR_UNSUPPORTED; }
+    h->use_tc = false;
+  }
+
+  seg_status st = SEG_OK;
+  auto bail = [&](seg_status s) { seg_destroy(h); return s; };
+
+  int64_t off = 0;
+  for (int l = 0; l < h->n_layers; ++l) {
+    LayerInfo L;
+    L.in = h->widths[l]; L.out = h->widths[l + 1];
+    L.ldw = round_up(L.in, 8);
+    L.w_off = off; off = round_up(off + (int64_t)L.out * L.ldw, 64);
+    L.b_off = off; off = round_up(off + L.out, 64);
+    h->layers.push_back(L);
+  }
+  h->n_flat = off;
+  if ((st = dev_alloc(h, &h->params, h->n_flat, true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->grads, h->n_flat, true)) != SEG_OK) return bail(st);
+  if (h->optimizer != SEG_SGD && (st = dev_alloc(h, &h->state1, h->n_flat, true)) != SEG_OK) return bail(st);
+  if (h->optimizer == SEG_ADAM && (st = dev_alloc(h, &h->state2, h->n_flat, true)) != SEG_OK) return bail(st);
+  if (h->precision != SEG_FP32) {
+    char* p = nullptr;
+    if ((st = dev_alloc(h, &p, h->n_flat * elem_size(h->op_dt), true)) != SEG_OK) return bail(st);
+    h->params_op = p;
+  }
+  h->act.assign(h->n_layers + 1, nullptr);
+  h->ld_act.assign(h->n_layers + 1, 0);
+  h->act_dtype.assign(h->n_layers + 1, h->act_dt);
+  int64_t max_ld = 0;
+  for (int l = 0; l <= h->n_layers; ++l) {
+    h->ld_act[l] = round_up(h->widths[l], 8);
+    if (l >= 1 && h->ld_act[l] > max_ld) max_ld = h->ld_act[l];
+  }
+  if (h->is_final) h->act_dtype[h->n_layers] = DT_F32;
+  for (int l = 1; l <= h->n_layers; ++l) {
+    char* p = nullptr;
+    const size_t bytes = (size_t)h->max_batch * h->ld_act[l] * elem_size(h->act_dtype[l]);
+    if ((st = dev_alloc(h, &p, bytes, true)) != SEG_OK) return bail(st);
+    h->act[l] = p;
+  }
+  {
+    char* p = nullptr;
+    if ((st = dev_alloc(h, &p, (size_t)h->max_batch * h->ld_act[0] * elem_size(h->act_dt), true)) != SEG_OK) return bail(st);
+    h->x_stage = p;
+  }
+  for (int i = 0; i < 2; ++i) {
+    if (i == 1 && h->n_layers == 1) break;
+    char* p = nullptr;
+    if ((st = dev_alloc(h, &p, (size_t)h->max_batch * max_ld * elem_size(h->act_dt), true)) != SEG_OK) return bail(st);
+    h->dz[i] = p;
+  }
+  if (!h->is_final &&
+      (st = dev_alloc(h, &h->sil, (size_t)h->n_classes * h->widths[h->n_layers], true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->loss_partials, loss_max_partials(), true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->loss_counter, 1, true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->dev_status, 1, true)) != SEG_OK) return bail(st);
+  if (cudaEventCreate(&h->ev_start) != cudaSuccess || cudaEventCreate(&h->ev_stop) != cudaSuccess)
+    return bail(SEG_ERR_CUDA);
+
+  for (int l = 0; l < h->n_layers; ++l) {
+    const LayerInfo& L = h->layers[l];
+    const float bound = 1.0f / sqrtf((float)L.in);
+    ++h->launches;
+    if (launch_init_uniform(h->params + L.w_off, L.out, L.in, L.ldw, h->init_seed, h->segment_id, l, 1,
+                            bound, h->stream) != cudaSuccess) return bail(SEG_ERR_CUDA);
+    ++h->launches;
+    if (launch_init_uniform(h->params + L.b_off, 1, L.out, L.out, h->init_seed, h->segment_id, l, 2,
+                            bound, h->stream) != cudaSuccess) return bail(SEG_ERR_CUDA);
+  }
+  if ((st = refresh_operand_copy(h, 0, h->n_flat)) != SEG_OK) return bail(st);
+  *out = h;
+  return SEG_OK;
+}
+
+seg_status seg_destroy(seg_handle* h) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  cudaStreamSynchronize(h->stream);
+  for (void* p : h->allocations) cudaFree(p);
+  for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+  if (h->ev_start) cudaEventDestroy(h->ev_start);
+  if (h->ev_stop) cudaEventDestroy(h->ev_stop);
+  cudaGetLastError();
+  delete h;
+  return SEG_OK;
+}
+
+seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, float kappa) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (h->is_final) return SEG_ERR_STATE;
+  if (dist != SEG_LABEL_UNIFORM_KAPPA && dist != SEG_LABEL_NORMAL) return SEG_ERR_INVALID_ARG;
+  Launch l(h, K_COPY);
+  SEG_TRY(h, launch_gen_labels(h->sil, h->n_classes, h->widths[h->n_layers], seed, h->segment_id, dist,
+                               kappa, h->stream), "label generation");
+  h->have_labels = true;
+  return SEG_OK;
+}
+
+seg_status seg_forward(seg_handle* h, const void* x, int32_t batch, void* y) {
+  if (!h || !x || !y) return SEG_ERR_INVALID_ARG;
+  if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
+  const void* x_use; int64_t ld_x;
+  seg_status st = forward_impl(h, x, batch, &x_use, &ld_x);
+  if (st != SEG_OK) return st;
+  return copy_out(h, y, batch);
+}
+
+seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
+                          float* loss_out, void* y_out) {
+  if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
+  if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
+  if (!h->is_final && !h->have_labels) return SEG_ERR_STATE;
+  const int L = h->n_layers;
+  const void* x_use; int64_t ld_x;   // where layer 0 read its input (the caller's x or the staged copy)
+  seg_status st = forward_impl(h, x, batch, &x_use, &ld_x);
+  if (st != SEG_OK) return st;
+  if (y_out && (st = copy_out(h, y_out, batch)) != SEG_OK) return st;
+
+  // loss -> dZ_L
+  void* dz_cur = h->dz[(L - 1) & 1];
+  {
+    Launch l(h, K_LOSS);
+    if (h->is_final) {
+      SEG_TRY(h, launch_softmax_ce_loss((const float*)h->act[L], h->ld_act[L], cls, h->n_classes, batch,
+                                        h->last_relu ? 1 : 0, dz_cur, h->act_dt, h->act_round, h->ld_act[L],
+                                        h->loss_partials, h->loss_counter, loss_out, h->stream), "softmax-CE loss");
+    } else {
+      SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], cls, h->sil, h->widths[L], batch,
+                                 h->last_relu ? 1 : 0, dz_cur, h->act_dt, h->act_round, h->ld_act[L],
+                                 h->loss_partials, h->loss_counter, loss_out, h->stream), "MSE loss");
+    }
+  }
+  // backward, layer by layer; dgrad of layer l is issued before anything overwrites W_l
+  for (int l = L - 1; l >= 0; --l) {
+    const LayerInfo& Ly = h->layers[l];
+    const int64_t ld_dz = h->ld_act[l + 1];
+    const void* a_prev = (l == 0) ? x_use : h->act[l];
+    const int64_t ld_prev = (l == 0) ? ld_x : h->ld_act[l];
+    {
+      Launch lb(h, K_BIAS);
+      SEG_TRY(h, launch_bias_grad(dz_cur, h->act_dt, ld_dz, batch, Ly.out, h->grads + Ly.b_off, nullptr,
+                                  h->stream), "bias gradient");
+    }
+    GemmDesc w{};
+    w.A = dz_cur; w.a_sm = 1; w.a_sk = ld_dz; w.a_dt = h->act_dt;
+    w.B = a_prev; w.b_sk = ld_prev; w.b_sn = 1; w.b_dt = h->act_dt;
+    w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
+    w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
+    if ((st = run_gemm(h, w, K_WGRAD)) != SEG_OK) return st;
+    if (l > 0) {
+      void* dz_next = h->dz[(l - 1) & 1];
+      GemmDesc d{};
+      d.A = dz_cur; d.a_sm = ld_dz; d.a_sk = 1; d.a_dt = h->act_dt;
+      d.B = weights_op(h, l); d.b_sk = Ly.ldw; d.b_sn = 1; d.b_dt = h->op_dt;
+      d.C = dz_next; d.ldc = h->ld_act[l]; d.c_dt = h->act_dt; d.c_round = h->act_round;
+      d.M = batch; d.N = Ly.in; d.K = Ly.out; d.epi = EPI_MASK;
+      d.mask = h->act[l]; d.ldmask = h->ld_act[l];
+      if ((st = run_gemm(h, d, K_DGRAD)) != SEG_OK) return st;
+      dz_cur = dz_next;
+    }
+  }
+  // optimizer
+  ++h->step;
+  UpdateArgs u{};
+  u.p = h->params; u.g = h->grads; u.s1 = h->state1; u.s2 = h->state2;
+  u.p_op = h->params_op; u.op_dt = h->op_dt; u.op_round = h->op_round;
+  u.n = h->n_flat; u.optimizer = h->optimizer;
+  u.lr = h->lr; u.momentum = h->momentum; u.beta1 = h->beta1; u.beta2 = h->beta2; u.eps = h->eps;
+  u.bc1 = (float)(1.0 - pow((double)h->beta1, (double)h->step));
+  u.bc2 = (float)(1.0 - pow((double)h->beta2, (double)h->step));
+  {
+    Launch lu(h, K_UPDATE);
+    SEG_TRY(h, launch_update(u, h->stream), "optimizer update");
+  }
+  return SEG_OK;
+}
+
+seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t* cls_host, int32_t batch,
+                               float* loss_host) {
+  if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
+  if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
+  seg_status st;
+  const size_t row_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
+  if (!h->host_x) {
+    char* p = nullptr;
+    if ((st = dev_alloc(h, &p, (size_t)h->max_batch * row_bytes, false)) != SEG_OK) return st;
+    h->host_x = p;
+    if ((st = dev_alloc(h, &h->host_cls, h->max_batch, false)) != SEG_OK) return st;
+    if ((st = dev_alloc(h, &h->host_loss, 1, true)) != SEG_OK) return st;
+  }
+  SEG_TRY(h, cudaMemcpyAsync(h->host_x, x_host, batch * row_bytes, cudaMemcpyHostToDevice, h->stream), "input copy");
+  SEG_TRY(h, cudaMemcpyAsync(h->host_cls, cls_host, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, h->stream), "class copy");
+  if ((st = seg_train_step(h, h->host_x, h->host_cls, batch, h->host_loss, nullptr)) != SEG_OK) return st;
+  if (loss_host)
+    SEG_TRY(h, cudaMemcpyAsync(loss_host, h->host_loss, sizeof(float), cudaMemcpyDeviceToHost, h->stream), "loss copy");
+  SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  return SEG_OK;
+}
+
+seg_status seg_get_labels(seg_handle* h, float* dst) {
+  if (!h || !dst) return SEG_ERR_INVALID_ARG;
+  if (h->is_final || !h->have_labels) return SEG_ERR_STATE;
+  SEG_TRY(h, cudaMemcpyAsync(dst, h->sil, sizeof(float) * h->n_classes * h->widths[h->n_layers],
+                             cudaMemcpyDeviceToDevice, h->stream), "label copy");
+  return SEG_OK;
+}
+
+seg_status seg_set_labels(seg_handle* h, const float* src) {
+  if (!h || !src) return SEG_ERR_INVALID_ARG;
+  if (h->is_final) return SEG_ERR_STATE;
+  SEG_TRY(h, cudaMemcpyAsync(h->sil, src, sizeof(float) * h->n_classes * h->widths[h->n_layers],
+                             cudaMemcpyDeviceToDevice, h->stream), "label copy");
+  h->have_labels = true;
+  return SEG_OK;
+}
+
+static seg_status get_flat(seg_handle* h, const float* base, int layer, float* W, float* b) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
+  if (!base) return SEG_ERR_STATE;
+  const LayerInfo& L = h->layers[layer];
+  if (W) {
+    Launch l(h, K_COPY);
+    SEG_TRY(h, launch_copy2d(W, DT_F32, L.in, base + L.w_off, DT_F32, L.ldw, L.out, L.in, RND_NONE, h->stream), "tensor copy");
+  }
+  if (b) SEG_TRY(h, cudaMemcpyAsync(b, base + L.b_off, sizeof(float) * L.out, cudaMemcpyDeviceToDevice, h->stream), "tensor copy");
+  return SEG_OK;
+}
+
+seg_status seg_get_params(seg_handle* h, int32_t layer, float* W, float* b) {
+  return get_flat(h, h ? h->params : nullptr, layer, W, b);
+}
+
+seg_status seg_get_grads(seg_handle* h, int32_t layer, float* dW, float* db) {
+  return get_flat(h, h ? h->grads : nullptr, layer, dW, db);
+}
+
+seg_status seg_get_opt_state(seg_handle* h, int32_t layer, int32_t which, float* sW, float* sb) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (which != 0 && which != 1) return SEG_ERR_INVALID_ARG;
+  return get_flat(h, which == 0 ? h->state1 : h->state2, layer, sW, sb);
+}
+
+seg_status seg_set_params(seg_handle* h, int32_t layer, const float* W, const float* b) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
+  const LayerInfo& L = h->layers[layer];
+  if (W) {
+    Launch l(h, K_COPY);
+    SEG_TRY(h, launch_copy2d(h->params + L.w_off, DT_F32, L.ldw, W, DT_F32, L.in, L.out, L.in, RND_NONE, h->stream), "tensor copy");
+  }
+  if (b) SEG_TRY(h, cudaMemcpyAsync(h->params + L.b_off, b, sizeof(float) * L.out, cudaMemcpyDeviceToDevice, h->stream), "tensor copy");
+  const int64_t end = (layer + 1 < h->n_layers) ? h->layers[layer + 1].w_off : h->n_flat;
+  return refresh_operand_copy(h, L.w_off, end - L.w_off);
+}
+
+seg_status seg_get_activation(seg_handle* h, int32_t layer, float* dst) {
+  if (!h || !dst) return SEG_ERR_INVALID_ARG;
+  if (layer < 1 || layer > h->n_layers) return SEG_ERR_SHAPE;
+  if (h->last_batch < 1) return SEG_ERR_STATE;
+  Launch l(h, K_COPY);
+  SEG_TRY(h, launch_copy2d(dst, DT_F32, h->widths[layer], h->act[layer], h->act_dtype[layer], h->ld_act[layer],
+                           h->last_batch, h->widths[layer], RND_NONE, h->stream), "activation copy");
+  return SEG_OK;
+}
+
+seg_status seg_mem_bytes(const seg_handle* h, uint64_t* current, uint64_t* peak) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (current) *current = h->mem_current;
+  if (peak) *peak = h->mem_peak;
+  return SEG_OK;
+}
+
+seg_status seg_launch_count(const seg_handle* h, uint64_t* launches) {
+  if (!h || !launches) return SEG_ERR_INVALID_ARG;
+  *launches = h->launches;
+  return SEG_OK;
+}
+
+seg_status seg_poll_status(seg_handle* h) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  int host = 0;
+  SEG_TRY(h, cudaMemcpyAsync(&host, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream), "status read");
+  SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  if (host != DEV_OK) {
+    cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream);
+    h->last_error = "a kernel gave up a bounded wait";
+    return SEG_ERR_DEVICE_TIMEOUT;
+  }
+  return SEG_OK;
+}
+
+seg_status seg_timer_start(seg_handle* h) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  SEG_TRY(h, cudaEventRecord(h->ev_start, h->stream), "event record");
+  return SEG_OK;
+}
+
+seg_status seg_timer_stop(seg_handle* h) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  SEG_TRY(h, cudaEventRecord(h->ev_stop, h->stream), "event record");
+  return SEG_OK;
+}
+
+seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms) {
+  if (!h || !ms) return SEG_ERR_INVALID_ARG;
+  SEG_TRY(h, cudaEventSynchronize(h->ev_stop), "event synchronize");
+  SEG_TRY(h, cudaEventElapsedTime(ms, h->ev_start, h->ev_stop), "event elapsed");
+  return SEG_OK;
+}
+
+seg_status seg_profile_enable(seg_handle* h, int32_t on) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  h->profile = on != 0;
+  h->ev_used = 0;
+  h->ev_kind.clear();
+  return SEG_OK;
+}
+
+seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms) {
+  if (!h || !count || !total_ms) return SEG_ERR_INVALID_ARG;
+  if (kind < 0 || kind >= K_COUNT) return SEG_ERR_INVALID_ARG;
+  SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  uint64_t n = 0; double total = 0.0;
+  for (size_t i = 0; i < h->ev_kind.size() && 2 * i + 1 < h->ev_used; ++i) {
+    if (h->ev_kind[i] != kind) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, h->ev_pool[2 * i], h->ev_pool[2 * i + 1]) == cudaSuccess) { total += ms; ++n; }
+  }
+  *count = n; *total_ms = (float)total;
+  return SEG_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+"""Helpers shared by the GPU parity tests: build the CUDA segment and the oracle segment from
+one description, feed both the same seeded arrays, and compare tensor by tensor."""
+import numpy as np
+
+from oracle import rng as orng
+from oracle.segment import OracleSegment
+from paper_2403_11204_b200 import workloads as wl
+
+
+def rel_err(got, ref):
+    """max |got - ref| / max |ref|  (element-wise ratios are meaningless next to ReLU zeros)."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.max(np.abs(got - ref)) / max(float(np.max(np.abs(ref))), 1e-30))
+
+
+DIST_CODE = {"uniform_kappa": orng.DIST_UNIFORM_KAPPA, "normal": orng.DIST_NORMAL}
+
+
+def make_pair(widths, n_classes, is_final, precision, optimizer, lr, max_batch, segment_id=0,
+              oracle_precision=None, gemm_backend="auto", label_dist="normal", kappa=10.0,
+              label_seed=wl.LABEL_SEED, init_seed=wl.INIT_SEED, momentum=0.9, last_relu=None):
+    from paper_2403_11204_b200.binding import Segment
+    gpu = Segment(widths, n_classes, is_final, precision=precision, optimizer=optimizer, lr=lr,
+                  momentum=momentum, max_batch=max_batch, segment_id=segment_id, init_seed=init_seed,
+                  gemm_backend=gemm_backend, last_relu=last_relu)
+    ora = OracleSegment(widths, n_classes, is_final, precision=oracle_precision or precision,
+                        optimizer=optimizer, lr=lr, momentum=momentum, segment_id=segment_id,
+                        init_seed=init_seed, last_relu=last_relu)
+    if not is_final:
+        gpu.gen_labels(label_seed, label_dist, kappa)
+        ora.gen_labels(label_seed, DIST_CODE[label_dist], kappa)
+    return gpu, ora
+
+
+def batch_arrays(workload, n, width, seed=wl.DATA_SEED, precision="fp32"):
+    x = wl.features(workload, n, width, seed)
+    cls = wl.class_indices(workload, n, seed)
+    if precision == "bf16":
+        x = wl.from_bf16_bits(wl.to_bf16_bits(x))      # both sides see bf16-representable inputs
+    return x, cls
+
+
+def to_device(x, cls, precision):
+    import torch
+    xt = torch.from_numpy(x).cuda()
+    if precision == "bf16":
+        xt = xt.to(torch.bfloat16)                       # exact: values are bf16-representable
+    return xt.contiguous(), torch.from_numpy(cls.astype(np.int32)).cuda()
+
+
+def bits_equal(a, b):
+    a = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    b = np.ascontiguousarray(b, dtype=np.float32).view(np.uint32)
+    return bool(np.array_equal(a, b))
+
+
+def compare_step(gpu, ora, x, cls, precision, tol, check_state=True):
+    """Runs one training step on both sides and returns {tensor name: relative error};
+    asserts every entry is within tol."""
+    import torch
+    xt, ct = to_device(x, cls, precision)
+    loss_t = torch.zeros(1, device="cuda")
+    gpu.train_step(xt, ct, loss_t)
+    gpu.poll()
+    loss_o = ora.train_step(x, cls)
+    errs = {"loss": abs(float(loss_t.item()) - loss_o) / max(abs(loss_o), 1e-30)}
+    for l in range(1, ora.n_layers + 1):
+        errs[f"A{l}"] = rel_err(gpu.activation(l).cpu().numpy(), ora.acts[l])
+    for l in range(ora.n_layers):
+        dW, db = gpu.grads(l)
+        errs[f"dW{l}"] = rel_err(dW.cpu().numpy(), ora.dW[l])
+        errs[f"db{l}"] = rel_err(db.cpu().numpy(), ora.db[l])
+        if check_state:
+            W, b = gpu.params(l)
+            errs[f"W{l}"] = rel_err(W.cpu().numpy(), ora.W[l])
+            errs[f"b{l}"] = rel_err(b.cpu().numpy(), ora.b[l])
+    bad = {k: v for k, v in errs.items() if not (v <= tol)}
+    assert not bad, f"beyond tolerance {tol}: {bad}  (all: {errs})"
+    return errs

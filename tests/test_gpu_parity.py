@@ -1,0 +1,158 @@
+"""CUDA path against the oracle, through the C ABI.  Tolerances (max |diff| / max |ref| per tensor):
+fp32 path 1e-4; TF32 path 1e-4 against the oracle that rounds where the kernels round and 2e-3
+against the unrounded fp32 oracle; bf16 path 2e-2."""
+import numpy as np
+import pytest
+
+from oracle import rng as orng
+from paper_2403_11204_b200 import workloads as wl
+from parity_util import batch_arrays, bits_equal, compare_step, make_pair, rel_err, to_device
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": 1e-4, "tf32": 1e-4, "bf16": 2e-2}
+
+
+# ---- (1) label generation and initialisation: bit-exact -----------------------------------
+@pytest.mark.parametrize("m,n_p", [(47, 64), (47, 60), (62, 2048), (3, 5), (1, 1), (1000, 1031)])
+@pytest.mark.parametrize("dist", ["uniform_kappa", "normal"])
+def test_labels_bit_exact(m, n_p, dist):
+    gpu, ora = make_pair([16, n_p], m, False, "fp32", "sgd", 0.01, 4, segment_id=3, label_dist=dist,
+                         label_seed=0x1234567890ABCDEF)
+    assert bits_equal(gpu.labels().cpu().numpy(), ora.sil)
+    gpu.close()
+
+
+def test_label_values_do_not_depend_on_other_handles_or_order():
+    a, ora = make_pair([8, 96], 10, False, "fp32", "sgd", 0.01, 4, segment_id=1)
+    b, _ = make_pair([8, 96], 10, False, "bf16", "adam", 0.01, 4, segment_id=1, gemm_backend="simt")
+    assert bits_equal(a.labels().cpu().numpy(), b.labels().cpu().numpy())
+    assert bits_equal(a.labels().cpu().numpy(), ora.sil)
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("widths", [[784, 128, 128, 64], [64, 64, 64, 47], [60, 60, 60, 47], [5, 3]])
+def test_initialisation_bit_exact(widths):
+    gpu, ora = make_pair(widths, 47, widths[-1] == 47, "fp32", "sgd", 0.01, 4, segment_id=2)
+    for l in range(ora.n_layers):
+        W, b = gpu.params(l)
+        assert bits_equal(W.cpu().numpy(), ora.W[l]) and bits_equal(b.cpu().numpy(), ora.b[l])
+    gpu.close()
+
+
+# ---- (2)-(4) one step: activations, loss, gradients, updated weights ----------------------------
+SMALL = [
+    # widths, final, precision, optimizer, batch
+    ([784, 128, 128, 64], False, "fp32", "sgd", 64),
+    ([64, 64, 64, 47], True, "fp32", "sgd", 64),
+    ([784, 80, 60], False, "fp32", "momentum", 141),
+    ([60, 60, 60, 47], True, "fp32", "momentum", 141),
+    ([100, 72, 40], False, "fp32", "adam", 33),
+    ([40, 24, 47], True, "fp32", "adam", 1),
+]
+
+
+@pytest.mark.parametrize("widths,final,precision,optimizer,batch", SMALL)
+def test_single_step_fp32(widths, final, precision, optimizer, batch):
+    w = wl.WORKLOADS["tiny"]
+    gpu, ora = make_pair(widths, 47, final, precision, optimizer, 0.01, batch)
+    x, cls = batch_arrays(w, batch, widths[0])
+    compare_step(gpu, ora, x, cls, precision, TOL[precision])
+    x2, cls2 = batch_arrays(w, batch, widths[0], seed=7)
+    compare_step(gpu, ora, x2, cls2, precision, TOL[precision])      # second step: optimizer state in play
+    gpu.close()
+
+
+@pytest.mark.parametrize("label_dist", ["uniform_kappa", "normal"])
+def test_tiny_workload_first_epoch_losses(label_dist):
+    """The tiny workload, segment 1: every batch of one epoch, loss by loss (fp32, SGD)."""
+    import torch
+    w = wl.WORKLOADS["tiny"]
+    spec = w.segments[0]
+    gpu, ora = make_pair(spec.widths, w.n_classes, False, "fp32", "sgd", w.lr, w.batch, label_dist=label_dist)
+    x, cls = batch_arrays(w, w.n_samples, spec.widths[0])
+    xt, ct = to_device(x, cls, "fp32")
+    losses = torch.zeros(w.n_samples // w.batch, device="cuda")
+    ref = []
+    for i in range(w.n_samples // w.batch):
+        sl = slice(i * w.batch, (i + 1) * w.batch)
+        gpu.train_step(xt[sl], ct[sl], losses[i:i + 1])
+        ref.append(ora.train_step(x[sl], cls[sl]))
+    gpu.poll()
+    got = losses.cpu().numpy()
+    assert np.max(np.abs(got - np.array(ref)) / np.abs(ref)) < 1e-4
+    gpu.close()
+
+
+REDUCED = [
+    ([96, 80, 64, 48], False, "tf32", "adam", 40),
+    ([48, 64, 32, 47], True, "tf32", "adam", 40),
+    ([96, 80, 64, 48], False, "bf16", "adam", 40),
+    ([48, 64, 32, 47], True, "bf16", "momentum", 40),
+    ([784, 256, 128, 64], False, "bf16", "sgd", 200),
+]
+
+
+@pytest.mark.parametrize("widths,final,precision,optimizer,batch", REDUCED)
+def test_single_step_reduced_precision_simt_backend(widths, final, precision, optimizer, batch):
+    """Rounding points of the TF32 / bf16 modes, run on the FFMA kernels."""
+    w = wl.WORKLOADS["tiny"]
+    gpu, ora = make_pair(widths, 47, final, precision, optimizer, 1e-3, batch, gemm_backend="simt")
+    x, cls = batch_arrays(w, batch, widths[0], precision=precision)
+    compare_step(gpu, ora, x, cls, precision, TOL[precision])
+    gpu.close()
+
+
+def test_forward_only_and_set_params_route():
+    import torch
+    w = wl.WORKLOADS["tiny"]
+    gpu, ora = make_pair([784, 128, 128, 64], 47, False, "fp32", "sgd", 0.01, 64, init_seed=11)
+    g = np.random.default_rng(0)
+    for l in range(ora.n_layers):                          # inject other weights on both sides
+        ora.W[l] = (g.standard_normal(ora.W[l].shape) * 0.05).astype(np.float32)
+        ora.b[l] = (g.standard_normal(ora.b[l].shape) * 0.05).astype(np.float32)
+        gpu.set_params(l, torch.from_numpy(ora.W[l]).cuda(), torch.from_numpy(ora.b[l]).cuda())
+    x, cls = batch_arrays(w, 50, 784)
+    xt, _ = to_device(x, cls, "fp32")
+    y = gpu.forward(xt)
+    gpu.poll()
+    assert rel_err(y.cpu().numpy(), ora.forward(x)[-1]) < 1e-4
+    gpu.close()
+
+
+def test_host_buffer_step_matches_device_step():
+    import torch
+    w = wl.WORKLOADS["tiny"]
+    a, ora = make_pair([784, 128, 128, 64], 47, False, "fp32", "sgd", 0.01, 64)
+    x, cls = batch_arrays(w, 64, 784)
+    loss = a.train_step_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(cls.astype(np.int32)).pin_memory())
+    ref = ora.train_step(x, cls)
+    assert abs(loss - ref) / abs(ref) < 1e-4
+    W, _ = a.params(0)
+    assert rel_err(W.cpu().numpy(), ora.W[0]) < 1e-4
+    a.close()
+
+
+def test_argument_errors_and_state():
+    import torch
+    from paper_2403_11204_b200.binding import SegError, Segment
+    seg = Segment([16, 8], 4, False, max_batch=8)
+    x = torch.zeros(4, 16, device="cuda")
+    c = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(SegError) as e:
+        seg.train_step(x, c)                               # labels never generated
+    assert e.value.status == 6
+    seg.gen_labels(1)
+    with pytest.raises(SegError) as e:
+        seg.train_step(torch.zeros(9, 16, device="cuda"), torch.zeros(9, dtype=torch.int32, device="cuda"))
+    assert e.value.status == 2                             # batch > max_batch
+    seg.train_step(x, c)
+    seg.poll()
+    cur, peak = seg.mem_bytes()
+    assert 0 < cur <= peak
+    assert seg.launch_count() > 0
+    seg.close()
+    fin = Segment([16, 4], 4, True, max_batch=8)
+    with pytest.raises(SegError):
+        fin.gen_labels(1)                                  # the final segment has no intermediate labels
+    fin.close()
