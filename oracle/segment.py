@@ -21,8 +21,9 @@ What is computed (paper: Section 2 for the procedure, Section 3 for the network)
 Precision modes
   "fp64": everything float64 (finite-difference checks).
   "fp32": fp32 storage of parameters/activations/gradients, float64 accumulation.
-  "tf32": as "fp32", with both operands of every matrix product rounded to TF32
-          (10-bit mantissa, round to nearest even) before the product.
+  "tf32": fp32 storage; matrix-product operands are TF32 (10-bit mantissa, round to
+          nearest even): weights through a rounded copy, hidden activations and
+          back-propagated dZ rounded when they are stored; final logits stay fp32.
   "bf16": fp32 master parameters; matrix-product operands are bf16: weights are rounded
           to bf16 copies, hidden activations and back-propagated dZ are stored in bf16;
           the final segment's logits stay fp32.
@@ -114,7 +115,11 @@ class OracleSegment:
 
     def _store_act(self, a64):
         a = a64.astype(self.store)
-        return round_bf16(a) if self.precision == "bf16" else a
+        if self.precision == "bf16":
+            return round_bf16(a)
+        if self.precision == "tf32":
+            return round_tf32(a)
+        return a
 
     # -- forward (Section 3: Linear + ReLU, identity on the network's last layer) -------
     def forward(self, x):

@@ -1,6 +1,526 @@
-// placeholder: tensor-core path
+// Tensor-core matrix products for sm_100a: TMA -> shared memory -> tcgen05.mma -> TMEM -> epilogue.
+//
+// One persistent, warp-specialised kernel serves the three products of a Linear layer:
+//   forward  C = A W^T     : both operands K-major (contraction index contiguous in memory)
+//   dgrad    C = dZ W      : A K-major, B MN-major
+//   wgrad    C = dZ^T A    : both operands MN-major (contraction over the batch)
+// with bf16 operands (kind::f16) or TF32 operands (kind::tf32) and fp32 accumulation in TMEM.
+//
+// CTA = 6 warps.  Warp 0 lane 0 issues TMA loads into a ring of shared-memory stages; warp 1 owns
+// the TMEM allocation and its lane 0 issues the MMAs; warps 2..5 drain the accumulator (each warp
+// reads its own 32 TMEM lanes), apply the epilogue and store.  Two accumulator buffers in TMEM let
+// the epilogue of tile i overlap the main loop of tile i+1.
+//
+// Shared-memory operand tiles use the 128-byte swizzle.  K-major tile: rows of 128 bytes (64 bf16
+// or 32 TF32 along K), 8-row groups 1024 bytes apart.  MN-major tile: chunks of 64 bf16 / 32 TF32
+// along M or N; inside a chunk each K index is one 128-byte row, 8-row groups 1024 bytes apart;
+// chunks follow each other at BLOCK_K * 128 bytes.
+//
+// Every wait on an mbarrier is bounded: after about two seconds the waiting thread raises an abort
+// flag, records DEV_TIMEOUT in the status word and all roles leave their loops; TMEM is released
+// before the CTA exits.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace segk {
-bool gemm_tc_init() { return false; }
-cudaError_t launch_gemm_tc(const GemmDesc&, int*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int TILE_ROW_BYTES = 128;                    // one swizzle row
+constexpr int A_TILE_BYTES = BLOCK_M * TILE_ROW_BYTES; // 16 KiB per stage
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BUDGET = 192 * 1024;                // operand ring
+constexpr int SMEM_EXTRA = 2048;                       // alignment slack + barriers
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the wait was abandoned (own time-out or another role's abort).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* dev_status) {
+  uint32_t spins = 0;
+  uint64_t t0 = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0xFFu) == 0u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicExch(dev_status, (int)DEV_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+template <bool TF32>
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  if constexpr (TF32) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
+// 32 lanes x 32 columns of fp32: thread i of the warp receives row (lane base + i), 32 columns.
+__device__ __forceinline__ void tmem_load_32x32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
+// in 16-byte units, descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+
+struct EpilogueArgs {
+  void* C;
+  int64_t ldc;
+  int c_dt, c_round, epi, relu;
+  const float* bias;
+  const void* mask;
+  int64_t ldmask;
+};
+
+template <int BLOCK_N>
+struct SmemLayout {
+  static constexpr int B_TILE_BYTES = BLOCK_N * TILE_ROW_BYTES;
+  static constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
+  static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
+  static constexpr int TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
+};
+
+// Epilogue for 32 consecutive columns of one row.
+__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], int row, int col0,
+                                               int n_total) {
+  const int n_valid = min(32, n_total - col0);
+  if (e.epi == EPI_BIAS_ACT) {
+    if (n_valid == 32) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        const float4 b = __ldg(reinterpret_cast<const float4*>(e.bias + col0 + j));
+        v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __ldg(e.bias + col0 + j);
+    }
+    if (e.relu) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+    }
+  } else if (e.epi == EPI_MASK) {
+    if (e.c_dt == DT_BF16) {
+      const __nv_bfloat16* mrow = reinterpret_cast<const __nv_bfloat16*>(e.mask) + (int64_t)row * e.ldmask + col0;
+      if (n_valid == 32) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          const uint4 q = __ldg(reinterpret_cast<const uint4*>(mrow + j));
+          const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            // a bf16 is positive iff its sign bit is clear and it is not zero
+            const uint32_t lo = w[t] & 0xFFFFu, hi = w[t] >> 16;
+            if (!(lo != 0u && lo < 0x8000u)) v[j + 2 * t] = 0.f;
+            if (!(hi != 0u && hi < 0x8000u)) v[j + 2 * t + 1] = 0.f;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (j < n_valid && !(__bfloat162float(mrow[j]) > 0.f)) v[j] = 0.f;
+      }
+    } else {
+      const float* mrow = reinterpret_cast<const float*>(e.mask) + (int64_t)row * e.ldmask + col0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid && !(__ldg(mrow + j) > 0.f)) v[j] = 0.f;
+    }
+  }
+  if (e.c_round == RND_TF32) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = round_tf32_rne(v[j]);
+  }
+  if (e.c_dt == DT_BF16) {
+    __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(e.C) + (int64_t)row * e.ldc + col0;
+    if (n_valid == 32 && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint4 q;
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]);
+        __nv_bfloat162 p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
+        __nv_bfloat162 p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+        q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
+        q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
+        *reinterpret_cast<uint4*>(crow + j) = q;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j < n_valid) crow[j] = __float2bfloat16_rn(v[j]);
+    }
+  } else {
+    float* crow = reinterpret_cast<float*>(e.C) + (int64_t)row * e.ldc + col0;
+    if (n_valid == 32 && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4)
+        *reinterpret_cast<float4*>(crow + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j < n_valid) crow[j] = v[j];
+    }
+  }
+}
+
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               int M, int N, int K, EpilogueArgs epi, int* dev_status) {
+  using L = SmemLayout<BLOCK_N>;
+  constexpr int STAGES = L::STAGES;
+  constexpr int BLOCK_K = TF32 ? 32 : 64;          // elements per stage along K (128 bytes K-major)
+  constexpr int UMMA_K = TF32 ? 8 : 16;            // elements per MMA along K (32 bytes)
+  constexpr int CHUNK = TF32 ? 32 : 64;            // elements per 128-byte row along M/N (MN-major)
+  constexpr int MN_CHUNK_BYTES = BLOCK_K * TILE_ROW_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * A_TILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * L::STAGE_BYTES);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
+  const int tiles_n = (N + BLOCK_N - 1) / BLOCK_N;
+  const int n_tiles = tiles_m * tiles_n;
+  const int num_k = (K + BLOCK_K - 1) / BLOCK_K;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        const int m0 = (t % tiles_m) * BLOCK_M, n0 = (t / tiles_m) * BLOCK_N;
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::STAGE_BYTES);
+          const uint32_t a_dst = smem_u32(smem_a + stage * A_TILE_BYTES);
+          const uint32_t b_dst = smem_u32(smem_b + stage * L::B_TILE_BYTES);
+          const int k0 = kb * BLOCK_K;
+          if constexpr (A_MN) {
+#pragma unroll
+            for (int c = 0; c < BLOCK_M / CHUNK; ++c)
+              tma_load_2d(a_dst + c * MN_CHUNK_BYTES, &map_a, m0 + c * CHUNK, k0, full_bar(stage));
+          } else {
+            tma_load_2d(a_dst, &map_a, k0, m0, full_bar(stage));
+          }
+          if constexpr (B_MN) {
+#pragma unroll
+            for (int c = 0; c < BLOCK_N / CHUNK; ++c)
+              tma_load_2d(b_dst + c * MN_CHUNK_BYTES, &map_b, n0 + c * CHUNK, k0, full_bar(stage));
+          } else {
+            tma_load_2d(b_dst, &map_b, k0, n0, full_bar(stage));
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, operand format, operand majors, N, M
+      constexpr uint32_t fmt = TF32 ? 2u : 1u;
+      constexpr uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BLOCK_N >> 3) << 17) |
+                                 ((uint32_t)(BLOCK_M >> 4) << 24);
+      constexpr uint32_t a_lbo = A_MN ? MN_CHUNK_BYTES : 16, b_lbo = B_MN ? MN_CHUNK_BYTES : 16;
+      constexpr uint32_t a_kstep = A_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      constexpr uint32_t b_kstep = B_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, dev_status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = smem_u32(smem_a + stage * A_TILE_BYTES);
+          const uint32_t b_src = smem_u32(smem_b + stage * L::B_TILE_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
+            const uint64_t da = make_smem_desc(a_src + kk * a_kstep, a_lbo, 1024);
+            const uint64_t db = make_smem_desc(b_src + kk * b_kstep, b_lbo, 1024);
+            tc_mma<TF32>(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));     // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));         // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int quarter = warp & 3;          // TMEM lanes 32*quarter .. +31 belong to this warp
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const int m0 = (t % tiles_m) * BLOCK_M, n0 = (t / tiles_m) * BLOCK_N;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+#pragma unroll 1
+      for (int c = 0; c < BLOCK_N / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= N) break;              // uniform across the CTA
+        float v[32];
+        tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
+        if (row < M) epilogue_store(epi, v, row, col0, N);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  if (*abort_flag) {
+    // give copies and MMAs still in flight time to land before shared memory and TMEM are released
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int g_num_sms = 0;
+bool g_init_done = false, g_init_ok = false;
+
+// 2-D tensor map over a row-major matrix: `inner` contiguous elements per row, `outer` rows,
+// `row_stride_bytes` between rows; box = box_inner x box_outer; 128-byte swizzle; zero fill.
+bool make_map(CUtensorMap* map, bool f32, const void* base, uint64_t inner, uint64_t outer,
+              uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {row_stride_bytes};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
+cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
+                           const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
+  using L = SmemLayout<BLOCK_N>;
+  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
+    if (err != cudaSuccess) return err;
+    attr_set = true;
+  }
+  const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + BLOCK_N - 1) / BLOCK_N);
+  const int grid = tiles < g_num_sms ? tiles : g_num_sms;
+  kern<<<grid, NUM_THREADS, L::TOTAL, s>>>(ma, mb, g.M, g.N, g.K, e, dev_status);
+  return cudaGetLastError();
+}
+
+template <bool TF32, int BLOCK_N>
+cudaError_t launch_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUtensorMap& mb,
+                          const GemmDesc& g, const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
+  if (!a_mn && !b_mn) return launch_variant<TF32, false, false, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  if (!a_mn && b_mn) return launch_variant<TF32, false, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  if (a_mn && b_mn) return launch_variant<TF32, true, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  return cudaErrorNotSupported;
+}
+
+int pick_block_n(int M, int N) {
+  const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
+  int best = 64; long best_cost = -1;
+  for (int bn : {256, 128, 64}) {
+    if (bn > 64 && bn / 2 >= N) continue;                  // do not use a tile twice as wide as N
+    const long tiles = (long)tiles_m * ((N + bn - 1) / bn);
+    const long waves = (tiles + g_num_sms - 1) / g_num_sms;
+    const long cost = waves * (bn + 32);                   // +32: per-tile fixed overhead
+    if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+  }
+  return best;
+}
+
+}  // namespace
+
+bool gemm_tc_init() {
+  if (g_init_done) return g_init_ok;
+  g_init_done = true;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    cudaGetLastError();
+    return false;
+  }
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  g_init_ok = g_num_sms > 0;
+  return g_init_ok;
+}
+
+cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
+  if (!g_init_ok) return cudaErrorNotSupported;
+  if (g.M <= 0 || g.N <= 0 || g.K <= 0) return cudaErrorNotSupported;
+  if (g.a_dt != g.b_dt) return cudaErrorNotSupported;
+  const bool tf32 = (g.a_dt == DT_F32);
+  const int esz = tf32 ? 4 : 2;
+  // operand majors from the strides
+  bool a_mn, b_mn;
+  int64_t a_pitch, b_pitch;
+  if (g.a_sk == 1) { a_mn = false; a_pitch = g.a_sm; }
+  else if (g.a_sm == 1) { a_mn = true; a_pitch = g.a_sk; }
+  else return cudaErrorNotSupported;
+  if (g.b_sk == 1) { b_mn = false; b_pitch = g.b_sn; }
+  else if (g.b_sn == 1) { b_mn = true; b_pitch = g.b_sk; }
+  else return cudaErrorNotSupported;
+  if (a_mn && !b_mn) return cudaErrorNotSupported;
+  // TMA rules: 16-byte aligned base, row pitch a multiple of 16 bytes
+  if ((reinterpret_cast<uintptr_t>(g.A) & 15u) || (reinterpret_cast<uintptr_t>(g.B) & 15u)) return cudaErrorNotSupported;
+  if ((a_pitch * esz) % 16 != 0 || (b_pitch * esz) % 16 != 0) return cudaErrorNotSupported;
+  if (a_pitch * (int64_t)esz >= (1ll << 40) || b_pitch * (int64_t)esz >= (1ll << 40)) return cudaErrorNotSupported;
+
+  const int block_n = pick_block_n(g.M, g.N);
+  const uint32_t block_k = tf32 ? 32 : 64, chunk = tf32 ? 32 : 64;
+  CUtensorMap ma, mb;
+  bool ok;
+  if (!a_mn) ok = make_map(&ma, tf32, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)a_pitch * esz, block_k, BLOCK_M);
+  else ok = make_map(&ma, tf32, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)a_pitch * esz, chunk, block_k);
+  if (!ok) return cudaErrorNotSupported;
+  if (!b_mn) ok = make_map(&mb, tf32, g.B, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)b_pitch * esz, block_k, (uint32_t)block_n);
+  else ok = make_map(&mb, tf32, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)b_pitch * esz, chunk, block_k);
+  if (!ok) return cudaErrorNotSupported;
+
+  EpilogueArgs e;
+  e.C = g.C; e.ldc = g.ldc; e.c_dt = g.c_dt; e.c_round = g.c_round; e.epi = g.epi; e.relu = g.relu;
+  e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
+
+#define SEGK_TC(TF, BN) launch_majors<TF, BN>(a_mn, b_mn, ma, mb, g, e, dev_status, s)
+  if (tf32) {
+    if (block_n == 256) return SEGK_TC(true, 256);
+    if (block_n == 128) return SEGK_TC(true, 128);
+    return SEGK_TC(true, 64);
+  }
+  if (block_n == 256) return SEGK_TC(false, 256);
+  if (block_n == 128) return SEGK_TC(false, 128);
+  return SEGK_TC(false, 64);
+#undef SEGK_TC
+}
+
+}  // namespace segk

@@ -156,3 +156,28 @@ def test_argument_errors_and_state():
     with pytest.raises(SegError):
         fin.gen_labels(1)                                  # the final segment has no intermediate labels
     fin.close()
+
+
+# ---- tensor-core products (tcgen05) against the oracle -----------------------------------------
+TC_CASES = [
+    # widths, final, precision, optimizer, batch   (shapes chosen to span several tiles + ragged tails)
+    ([64, 128], False, "bf16", "sgd", 128),                 # one tile, forward + wgrad only
+    ([128, 256, 128], False, "bf16", "sgd", 256),           # adds dgrad
+    ([784, 320, 200, 72], False, "bf16", "adam", 300),      # K tail (784), ragged M / N
+    ([72, 136, 264, 47], True, "bf16", "momentum", 129),    # final segment, 47 logits in fp32
+    ([1024, 512, 512], False, "bf16", "adam", 1024),        # many tiles, several k blocks
+    ([64, 128], False, "tf32", "sgd", 128),
+    ([784, 320, 200, 72], False, "tf32", "adam", 300),
+    ([72, 136, 264, 47], True, "tf32", "adam", 129),
+]
+
+
+@pytest.mark.parametrize("widths,final,precision,optimizer,batch", TC_CASES)
+def test_single_step_tensor_core_backend(widths, final, precision, optimizer, batch):
+    w = wl.WORKLOADS["tiny"]
+    gpu, ora = make_pair(widths, 47, final, precision, optimizer, 1e-3, batch, gemm_backend="tcgen05")
+    x, cls = batch_arrays(w, batch, widths[0], precision=precision)
+    compare_step(gpu, ora, x, cls, precision, TOL[precision])
+    x2, cls2 = batch_arrays(w, batch - 1, widths[0], seed=5, precision=precision)
+    compare_step(gpu, ora, x2, cls2, precision, TOL[precision])      # smaller batch on the same handle
+    gpu.close()
