@@ -160,6 +160,13 @@ SEG_API seg_status seg_get_grads(seg_handle* h, int32_t layer, float* dW, float*
 /* Optimizer state of layer `layer`: which = 0 momentum buffer / Adam first moment,
  * which = 1 Adam second moment; shapes as the parameters.                                */
 SEG_API seg_status seg_get_opt_state(seg_handle* h, int32_t layer, int32_t which, float* sW, float* sb);
+SEG_API seg_status seg_set_opt_state(seg_handle* h, int32_t layer, int32_t which, const float* sW,
+                                     const float* sb);
+
+/* Number of optimizer steps taken (the t of Adam's bias correction); host pointer.  Setting it
+ * together with parameters and optimizer state resumes a saved segment.                     */
+SEG_API seg_status seg_get_step(const seg_handle* h, uint64_t* step);
+SEG_API seg_status seg_set_step(seg_handle* h, uint64_t step);
 
 /* Stored output A_layer of the last step, layer = 1..n_layers, converted to fp32
  * [batch][widths[layer]] for the batch size of that step.                                */

@@ -45,6 +45,9 @@ EXPORTS = {
     "seg_set_params": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p]),
     "seg_get_grads": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p]),
     "seg_get_opt_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
+    "seg_set_opt_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
+    "seg_get_step": (c_int32, [c_void_p, POINTER(c_uint64)]),
+    "seg_set_step": (c_int32, [c_void_p, c_uint64]),
     "seg_get_activation": (c_int32, [c_void_p, c_int32, c_void_p]),
     "seg_mem_bytes": (c_int32, [c_void_p, POINTER(c_uint64), POINTER(c_uint64)]),
     "seg_launch_count": (c_int32, [c_void_p, POINTER(c_uint64)]),
@@ -203,6 +206,20 @@ class Segment:
         b = b.contiguous().float()
         self._check(self.lib.seg_set_params(self.h, layer, _ptr(W), _ptr(b)), "seg_set_params")
         self.stream.synchronize()
+
+    def set_opt_state(self, layer, which, sW, sb):
+        sW = sW.contiguous().float()
+        sb = sb.contiguous().float()
+        self._check(self.lib.seg_set_opt_state(self.h, layer, which, _ptr(sW), _ptr(sb)), "seg_set_opt_state")
+        self.stream.synchronize()
+
+    def step_count(self):
+        n = c_uint64()
+        self._check(self.lib.seg_get_step(self.h, byref(n)), "seg_get_step")
+        return n.value
+
+    def set_step(self, t):
+        self._check(self.lib.seg_set_step(self.h, int(t)), "seg_set_step")
 
     def activation(self, layer):
         t = self._empty(self.last_batch, self.widths[layer])

@@ -13,8 +13,10 @@
 //
 // Shared-memory operand tiles use the 128-byte swizzle.  K-major tile: rows of 128 bytes (64 bf16
 // or 32 TF32 along K), 8-row groups 1024 bytes apart.  MN-major tile: chunks of 64 bf16 / 32 TF32
-// along M or N; inside a chunk each K index is one 128-byte row, 8-row groups 1024 bytes apart;
-// chunks follow each other at BLOCK_K * 128 bytes.
+// along M or N; inside a chunk each K index is one 128-byte row; chunks follow each other at
+// BLOCK_K * 128 bytes.  bf16 MN-major tiles use the ordinary 128-byte swizzle (16-byte atoms,
+// 8-row groups 1024 bytes apart); 32-bit MN-major tiles must use the 128-byte swizzle with
+// 32-byte atoms (4-row groups 512 bytes apart), in the tensor map and in the descriptor alike.
 //
 // Every wait on an mbarrier is bounded: after about two seconds the waiting thread raises an abort
 // flag, records DEV_TIMEOUT in the status word and all roles leave their loops; TMEM is released
@@ -132,13 +134,14 @@ __device__ __forceinline__ void tmem_load_32x32(uint32_t taddr, float (&v)[32]) 
 
 // Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
 // in 16-byte units, descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                   uint32_t layout_type) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= (uint64_t)1 << 46;   // descriptor version
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  d |= (uint64_t)layout_type << 61;   // 2: 128-byte swizzle; 1: 128-byte swizzle, 32-byte atoms
   return d;
 }
 
@@ -329,6 +332,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       constexpr uint32_t a_lbo = A_MN ? MN_CHUNK_BYTES : 16, b_lbo = B_MN ? MN_CHUNK_BYTES : 16;
       constexpr uint32_t a_kstep = A_MN ? UMMA_K * TILE_ROW_BYTES : 32;
       constexpr uint32_t b_kstep = B_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      // 32-bit MN-major operands: 32-byte-atom swizzle, groups of 4 K rows (512 bytes)
+      constexpr uint32_t a_sbo = (TF32 && A_MN) ? 512 : 1024, b_sbo = (TF32 && B_MN) ? 512 : 1024;
+      constexpr uint32_t a_lay = (TF32 && A_MN) ? 1 : 2, b_lay = (TF32 && B_MN) ? 1 : 2;
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
@@ -343,8 +349,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t b_src = smem_u32(smem_b + stage * L::B_TILE_BYTES);
 #pragma unroll
           for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
-            const uint64_t da = make_smem_desc(a_src + kk * a_kstep, a_lbo, 1024);
-            const uint64_t db = make_smem_desc(b_src + kk * b_kstep, b_lbo, 1024);
+            const uint64_t da = make_smem_desc(a_src + kk * a_kstep, a_lbo, a_sbo, a_lay);
+            const uint64_t db = make_smem_desc(b_src + kk * b_kstep, b_lbo, b_sbo, b_lay);
             tc_mma<TF32>(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));     // frees the stage once these MMAs have read it
@@ -402,16 +408,18 @@ int g_num_sms = 0;
 bool g_init_done = false, g_init_ok = false;
 
 // 2-D tensor map over a row-major matrix: `inner` contiguous elements per row, `outer` rows,
-// `row_stride_bytes` between rows; box = box_inner x box_outer; 128-byte swizzle; zero fill.
+// `row_stride_bytes` between rows; box = box_inner x box_outer; 128-byte swizzle (32-byte atoms
+// when atom32); zero fill.
 bool make_map(CUtensorMap* map, bool f32, const void* base, uint64_t inner, uint64_t outer,
-              uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer) {
+              uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, bool atom32) {
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {row_stride_bytes};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -500,11 +508,11 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   const uint32_t block_k = tf32 ? 32 : 64, chunk = tf32 ? 32 : 64;
   CUtensorMap ma, mb;
   bool ok;
-  if (!a_mn) ok = make_map(&ma, tf32, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)a_pitch * esz, block_k, BLOCK_M);
-  else ok = make_map(&ma, tf32, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)a_pitch * esz, chunk, block_k);
+  if (!a_mn) ok = make_map(&ma, tf32, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)a_pitch * esz, block_k, BLOCK_M, false);
+  else ok = make_map(&ma, tf32, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)a_pitch * esz, chunk, block_k, tf32);
   if (!ok) return cudaErrorNotSupported;
-  if (!b_mn) ok = make_map(&mb, tf32, g.B, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)b_pitch * esz, block_k, (uint32_t)block_n);
-  else ok = make_map(&mb, tf32, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)b_pitch * esz, chunk, block_k);
+  if (!b_mn) ok = make_map(&mb, tf32, g.B, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)b_pitch * esz, block_k, (uint32_t)block_n, false);
+  else ok = make_map(&mb, tf32, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)b_pitch * esz, chunk, block_k, tf32);
   if (!ok) return cudaErrorNotSupported;
 
   EpilogueArgs e;

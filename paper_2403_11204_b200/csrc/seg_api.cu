@@ -506,6 +506,33 @@ seg_status seg_get_opt_state(seg_handle* h, int32_t layer, int32_t which, float*
   return get_flat(h, which == 0 ? h->state1 : h->state2, layer, sW, sb);
 }
 
+seg_status seg_set_opt_state(seg_handle* h, int32_t layer, int32_t which, const float* sW, const float* sb) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (which != 0 && which != 1) return SEG_ERR_INVALID_ARG;
+  if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
+  float* base = which == 0 ? h->state1 : h->state2;
+  if (!base) return SEG_ERR_STATE;
+  const LayerInfo& L = h->layers[layer];
+  if (sW) {
+    Launch l(h, K_COPY);
+    SEG_TRY(h, launch_copy2d(base + L.w_off, DT_F32, L.ldw, sW, DT_F32, L.in, L.out, L.in, RND_NONE, h->stream), "tensor copy");
+  }
+  if (sb) SEG_TRY(h, cudaMemcpyAsync(base + L.b_off, sb, sizeof(float) * L.out, cudaMemcpyDeviceToDevice, h->stream), "tensor copy");
+  return SEG_OK;
+}
+
+seg_status seg_get_step(const seg_handle* h, uint64_t* step) {
+  if (!h || !step) return SEG_ERR_INVALID_ARG;
+  *step = h->step;
+  return SEG_OK;
+}
+
+seg_status seg_set_step(seg_handle* h, uint64_t step) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  h->step = step;
+  return SEG_OK;
+}
+
 seg_status seg_set_params(seg_handle* h, int32_t layer, const float* W, const float* b) {
   if (!h) return SEG_ERR_INVALID_ARG;
   if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
