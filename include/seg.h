@@ -197,6 +197,34 @@ SEG_API seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms);
 SEG_API seg_status seg_profile_enable(seg_handle* h, int32_t on);
 SEG_API seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms);
 
+/* The intermediate-label loss without any allocation (the paper has no counterpart: this
+ * entry point exists for the callers described below, not for the method).
+ *
+ * Some callers cannot allocate device memory: a plug-in running inside another program's
+ * fixed memory budget, a latency-bound loop where the device synchronisation that
+ * cudaMalloc implies is not acceptable, code that is given a stream and buffers but no
+ * allocator.  For them this call computes what a non-final segment's loss kernel computes -
+ *     loss = mean_{b,i} (out[b][i] - sil[cls[b]][i])^2,
+ *     dz[b][i] = 2 (out[b][i] - sil[cls[b]][i]) / (batch * n_p) * (relu_mask ? out[b][i] > 0 : 1)
+ * - without a handle and without calling cudaMalloc, cudaFree or any allocating routine.
+ * The reduction scratch is a static device array of 8 KiB inside the library, present on
+ * every GPU that loads the library until the process exits.
+ *   out [batch][n_p] float, cls [batch] int32 in [0, n_classes), sil [n_classes][n_p] float,
+ *   dz [batch][n_p] float (written), loss_out device float (written; may be NULL),
+ *   stream: cudaStream_t.  All device pointers, dense row-major, caller-owned.
+ * Limits: n_p <= SEG_NOALLOC_MAX_WIDTH, batch <= SEG_NOALLOC_MAX_BATCH; anything larger
+ * returns SEG_ERR_SHAPE and enqueues nothing.
+ * The first call on a device looks up the array's device address (once per device, with
+ * that device current); make that first call before starting any stream capture.
+ * Every call on a device shares the one array: calls whose kernels may overlap on the GPU
+ * (different streams, no dependency between them) race on it and give wrong losses; order
+ * them on one stream or with events.  Nothing needs clearing by the caller.               */
+#define SEG_NOALLOC_MAX_WIDTH 65536
+#define SEG_NOALLOC_MAX_BATCH 65536
+SEG_API seg_status seg_label_loss_noalloc(const float* out, const int32_t* cls, const float* sil,
+                                          int32_t n_classes, int32_t n_p, int32_t batch,
+                                          int32_t relu_mask, float* dz, float* loss_out, void* stream);
+
 SEG_API const char* seg_status_string(int32_t s);
 
 /* Text of the last CUDA error seen by this handle ("" if none); valid until the next call. */

@@ -57,6 +57,8 @@ EXPORTS = {
     "seg_timer_elapsed_ms": (c_int32, [c_void_p, POINTER(c_float)]),
     "seg_profile_enable": (c_int32, [c_void_p, c_int32]),
     "seg_profile_get": (c_int32, [c_void_p, c_int32, POINTER(c_uint64), POINTER(c_float)]),
+    "seg_label_loss_noalloc": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32,
+                                         c_void_p, c_void_p, c_void_p]),
     "seg_status_string": (c_char_p, [c_int32]),
     "seg_last_error": (c_char_p, [c_void_p]),
     "seg_build_info": (c_char_p, []),
@@ -89,6 +91,24 @@ class SegError(RuntimeError):
 
 def _ptr(t):
     return None if t is None else c_void_p(t.data_ptr())
+
+
+def label_loss_noalloc(out, cls, sil, relu_mask, dz, loss_out, stream=None):
+    """seg_label_loss_noalloc on torch CUDA tensors: the intermediate-label loss and its dZ for
+    callers that must not allocate device memory (the library's static scratch is used).
+    out [batch, n_p] fp32, cls [batch] int32, sil [n_classes, n_p] fp32; dz and loss_out are
+    written.  Calls that may overlap on the GPU share the scratch and must be ordered."""
+    import torch
+    lib = load()
+    for t in (out, cls, sil, dz):
+        assert t.is_cuda and t.is_contiguous()
+    assert out.dtype == torch.float32 and sil.dtype == torch.float32 and dz.dtype == torch.float32
+    assert cls.dtype == torch.int32 and dz.shape == out.shape and sil.shape[1] == out.shape[1]
+    st = stream if stream is not None else torch.cuda.current_stream()
+    status = lib.seg_label_loss_noalloc(_ptr(out), _ptr(cls), _ptr(sil), sil.shape[0], out.shape[1], out.shape[0],
+                                        int(bool(relu_mask)), _ptr(dz), _ptr(loss_out), c_void_p(st.cuda_stream))
+    if status != SEG_OK:
+        raise SegError(status, "seg_label_loss_noalloc")
 
 
 class Segment:

@@ -314,3 +314,62 @@ cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src
 }
 
 }  // namespace segk
+
+// ---- entry point that allocates nothing ---------------------------------------------------------
+// The intermediate-label loss for callers that may not allocate device memory: plug-ins that run
+// inside another program's fixed memory budget, latency-bound loops that cannot afford the device
+// synchronisation cudaMalloc implies, code that is handed a stream and buffers but no allocator.
+// The reduction scratch the loss kernel needs (one partial sum per thread block and the arrival
+// counter) lives in the file-scope device array below instead of a handle's workspace.  The array
+// exists once on every device that loads this library and is held until the process exits.
+namespace segk {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 8192;           // 1024 block partials (4 KiB) + arrival counter
+static __device__ __align__(256) unsigned char g_static_loss_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {};          // device address of the array, per device
+
+// In host code the array's name is only a handle for the runtime, not a device address; the
+// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that
+// device current.
+cudaError_t static_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_loss_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_scratch_ptr[dev] = p;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace segk
+
+extern "C" SEG_API seg_status seg_label_loss_noalloc(const float* out, const int32_t* cls, const float* sil,
+                                                     int32_t n_classes, int32_t n_p, int32_t batch,
+                                                     int32_t relu_mask, float* dz, float* loss_out,
+                                                     void* stream) {
+  using namespace segk;
+  if (!out || !cls || !sil || !dz) return SEG_ERR_INVALID_ARG;
+  if (n_classes < 1 || n_p < 1 || batch < 1) return SEG_ERR_SHAPE;
+  if (n_p > SEG_NOALLOC_MAX_WIDTH || batch > SEG_NOALLOC_MAX_BATCH) return SEG_ERR_SHAPE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  void* scratch = nullptr;
+  if (static_scratch_address(&scratch) != cudaSuccess) { cudaGetLastError(); return SEG_ERR_CUDA; }
+  float* partials = reinterpret_cast<float*>(scratch);
+  unsigned int* counter = reinterpret_cast<unsigned int*>(reinterpret_cast<unsigned char*>(scratch) + 4096);
+  // the array keeps whatever the previous call left: the arrival counter must start at zero
+  if (cudaMemsetAsync(counter, 0, sizeof(unsigned int), s) != cudaSuccess) { cudaGetLastError(); return SEG_ERR_CUDA; }
+  const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
+  mse_loss_kernel<float, float><<<grid, kLossThreads, 0, s>>>(out, n_p, cls, sil, n_p, batch, relu_mask ? 1 : 0, dz,
+                                                             RND_NONE, n_p, partials, counter, loss_out);
+  if (cudaGetLastError() != cudaSuccess) return SEG_ERR_CUDA;
+  return SEG_OK;
+}
