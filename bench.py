@@ -242,11 +242,13 @@ class Runner:
             seg.close()
 
 
-def measure(workload, steps, warmup, peaks, device_index=0, full=True):
+def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples=None):
     """Runs one workload.  full=True adds the end-to-end leg, per-kernel profile and clocks."""
     import torch
     w = workload
-    r = Runner(w, device_index, host_data=full, n_samples=None if full else min(w.n_samples, 64 * w.batch))
+    if n_samples is None and not full:
+        n_samples = min(w.n_samples, 64 * w.batch)
+    r = Runner(w, device_index, host_data=full, n_samples=n_samples)
     r.prepare()
     label_ms = r.gen_labels()
     r.materialise_inputs()
@@ -352,6 +354,7 @@ def main():
     ap.add_argument("--others", default="bf16_wide,gemm_large,multi_cut,tiny",
                     help="further workloads summarised in the same line ('' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--samples", type=int, default=0, help="size of the resident data set (0: the workload's own)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = wl.WORKLOADS[args.workload]
@@ -386,7 +389,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist.barrier()
     peaks = load_peaks()
-    res = measure(w, args.steps, args.warmup, peaks, device_index=local_rank, full=True)
+    res = measure(w, args.steps, args.warmup, peaks, device_index=local_rank, full=True,
+                  n_samples=args.samples or None)
     ms_total = res["ms_per_step"] * args.steps
     if world > 1:
         t = torch.tensor([ms_total], device="cuda")

@@ -27,6 +27,12 @@ Precision modes
   "bf16": fp32 master parameters; matrix-product operands are bf16: weights are rounded
           to bf16 copies, hidden activations and back-propagated dZ are stored in bf16;
           the final segment's logits stay fp32.
+ReLU ties.  relu'(z) is taken as 1 for z > 0 and 0 otherwise, decided on the oracle's own
+pre-activation.  A caller comparing against another implementation may pass `tie_break`
+to loss_and_grads: for elements whose |z| is below the caller's ambiguity threshold (both
+signs are correct answers within the stated tolerance of the activations) it may choose
+the derivative; everywhere else the oracle's own decision stands.  The forward values
+are never altered.
 Pins live in tests/test_oracle_segment.py (finite differences, closed forms, invariants).
 """
 import numpy as np
@@ -124,11 +130,13 @@ class OracleSegment:
     # -- forward (Section 3: Linear + ReLU, identity on the network's last layer) -------
     def forward(self, x):
         acts = [np.asarray(x, dtype=self.store)]
+        self.preact = []
         for l in range(self.n_layers):
             a_op = self._operand(acts[-1]).astype(np.float64)
             w_op = self._operand(self.W[l]).astype(np.float64)
             z = a_op @ w_op.T + self.b[l].astype(np.float64)
             last = l == self.n_layers - 1
+            self.preact.append(z)
             if (not last) or self.last_relu:
                 z = np.maximum(z, 0.0)
             if last and self.is_final:
@@ -138,18 +146,25 @@ class OracleSegment:
         return acts
 
     # -- loss + backward -------------------------------------------------------------
-    def loss_and_grads(self, x, cls):
+    def loss_and_grads(self, x, cls, tie_break=None):
+        """tie_break(layer, z, mask) -> mask: optional choice of relu' on near-zero pre-activations
+        (layer = 1-based index of the activation A_layer, z = fp64 pre-activation, mask = z > 0)."""
         cls = np.asarray(cls, dtype=np.int64)
         acts = self.forward(x)
         out = acts[-1]
+        masks = [None] * (self.n_layers + 1)
+        for l in range(1, self.n_layers + 1):
+            if l < self.n_layers or self.last_relu:
+                m = acts[l] > 0
+                masks[l] = tie_break(l, self.preact[l - 1], m) if tie_break is not None else m
         if self.is_final:
             loss, dz = softmax_ce_loss(out, cls)
             if self.last_relu:
-                dz = dz * (out > 0)
+                dz = dz * masks[-1]
         else:
             target = self.sil[cls]                          # gather: one SIL row per sample
             loss, da = mse_loss(out, target)
-            dz = da * (out > 0) if self.last_relu else da   # relu'(0) taken as 0
+            dz = da * masks[-1] if self.last_relu else da   # relu'(0) taken as 0
         dZ = [None] * self.n_layers
         dW = [None] * self.n_layers
         db = [None] * self.n_layers
@@ -163,7 +178,7 @@ class OracleSegment:
             if l > 0:
                 w_op = self._operand(self.W[l]).astype(np.float64)
                 da_prev = dz_op @ w_op
-                dz = self._store_act(da_prev * (acts[l] > 0))
+                dz = self._store_act(da_prev * masks[l])
         self.acts, self.dZ, self.dW, self.db = acts, dZ, dW, db
         return loss
 
@@ -189,9 +204,9 @@ class OracleSegment:
                 new = p64 - self.lr * mhat / (np.sqrt(vhat) + self.eps)
             p[...] = new.astype(self.store)
 
-    def train_step(self, x, cls):
+    def train_step(self, x, cls, tie_break=None):
         """One step: forward, loss, backward, update.  Returns the loss before the update."""
-        loss = self.loss_and_grads(x, cls)
+        loss = self.loss_and_grads(x, cls, tie_break)
         self.apply_update()
         return loss
 

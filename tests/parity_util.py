@@ -79,16 +79,34 @@ def compare_step(gpu, ora, x, cls, precision, tol, check_state=True):
     error the updated weight is ill-conditioned: two correct gradients within tolerance of each
     other give updates that differ by up to 2 lr.  There the comparison is made on the elements
     whose reference gradient is at least ten times the measured gradient error (same tolerance),
-    and every other element is held to the absolute bound 3 lr that Adam's step size implies."""
+    and every other element is held to the absolute bound 3 lr that Adam's step size implies.
+
+    ReLU ties: relu' is a decision taken from a floating-point value.  Where the oracle's own
+    pre-activation is within 5 % of the activation tolerance of zero, both derivatives are correct
+    answers (an output within tolerance may sit on either side of zero), so there the oracle's
+    backward pass follows the sign the CUDA path stored (which must itself be that small); everywhere
+    else the oracle decides alone and the stored signs must agree with it."""
     import torch
     xt, ct = to_device(x, cls, precision)
     loss_t = torch.zeros(1, device="cuda")
     gpu.train_step(xt, ct, loss_t)
     gpu.poll()
-    loss_o = ora.train_step(x, cls)
+    acts_gpu = {l: gpu.activation(l).cpu().numpy() for l in range(1, ora.n_layers + 1)}
+    ties = {}
+
+    def tie_break(l, z, m):
+        thr = 0.05 * tol * max(float(np.max(z)), 1e-30)
+        amb = np.abs(z) <= thr
+        g_on = acts_gpu[l] > 0
+        assert float(np.max(np.abs(acts_gpu[l][amb]), initial=0.0)) <= 2.0 * thr, f"A{l}: large value at a tie"
+        assert np.array_equal(g_on[~amb], m[~amb]), f"A{l}: ReLU sign differs away from zero"
+        ties[l] = float(np.mean(amb & (g_on != m)))
+        return np.where(amb, g_on, m)
+
+    loss_o = ora.train_step(x, cls, tie_break)
     errs = {"loss": abs(float(loss_t.item()) - loss_o) / max(abs(loss_o), 1e-30)}
     for l in range(1, ora.n_layers + 1):
-        errs[f"A{l}"] = rel_err(gpu.activation(l).cpu().numpy(), ora.acts[l])
+        errs[f"A{l}"] = rel_err(acts_gpu[l], ora.acts[l])
     for l in range(ora.n_layers):
         dW, db = (t.cpu().numpy() for t in gpu.grads(l))
         errs[f"dW{l}"] = rel_err(dW, ora.dW[l])

@@ -267,3 +267,37 @@ def test_reduced_precision_modes_stay_close_to_fp32_mode():
         seg.loss_and_grads(x, cls)
         for a, b in zip(ref.dW + ref.db + ref.acts[1:], seg.dW + seg.db + seg.acts[1:]):
             assert np.max(np.abs(a.astype(np.float64) - b)) <= tol * np.max(np.abs(a))
+
+
+def test_tie_break_only_acts_where_the_caller_flips_and_matches_a_perturbed_network():
+    """Choosing relu' = 0 on one barely-positive unit equals the gradient of the same network with that
+    unit's bias lowered by more than its pre-activation (the unit is then off, the forward output of
+    everything else unchanged up to that tiny amount)."""
+    seg = make([6, 5, 4], False, n_classes=3)
+    x, cls = data(seg, 4, seed=11)
+    seg.forward(x)
+    z = seg.preact[0]
+    b_idx, j = np.unravel_index(np.argmin(np.where(z > 0, z, np.inf)), z.shape)   # smallest positive unit
+    eps = float(z[b_idx, j])
+    base = seg.loss_and_grads(x, cls)
+    g_plain = [g.copy() for g in seg.dW + seg.db]
+    same = seg.loss_and_grads(x, cls, tie_break=lambda l, zz, m: m)
+    assert same == base and all(np.array_equal(a, b) for a, b in zip(g_plain, seg.dW + seg.db))
+
+    def flip(l, zz, m):
+        m = m.copy()
+        if l == 1:
+            m[b_idx, j] = False
+        return m
+    seg.loss_and_grads(x, cls, tie_break=flip)
+    g_flip = [g.copy() for g in seg.dW + seg.db]
+    other = make([6, 5, 4], False, n_classes=3)
+    xs = x.copy()
+    # switch the unit off for that sample only: subtract from the sample's input what lowers z by 2*eps
+    w = other.W[0][j]
+    xs[b_idx] = xs[b_idx] - 2 * eps * w / float(w @ w)
+    other.loss_and_grads(xs, cls)
+    assert (other.preact[0][b_idx, j] < 0) and np.sum((other.preact[0] > 0) != (z > 0)) == 1
+    for a, b in zip(g_flip, other.dW + other.db):
+        assert np.allclose(a, b, atol=20 * eps * (1 + np.abs(b).max()) + 1e-12)
+    assert any(not np.array_equal(a, b) for a, b in zip(g_flip, g_plain))
