@@ -65,8 +65,9 @@ int loss_max_partials();
 
 // db[n] = sum_b dZ[b][n], deterministic
 cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, int n, float* db,
-                             float* scratch, cudaStream_t s);
-int bias_grad_scratch_floats(int batch, int n);
+                             float* partials, unsigned int* counters, cudaStream_t s);
+int bias_grad_partial_floats(int batch, int n);
+int bias_grad_counters(int n);
 
 struct UpdateArgs {
   float* p; const float* g; float* s1; float* s2;
@@ -76,13 +77,18 @@ struct UpdateArgs {
   int64_t n;
   int optimizer;
   float lr, momentum, beta1, beta2, eps;
-  float bc1, bc2;      // Adam bias corrections 1-b1^t, 1-b2^t
+  const float* bc;     // device: {1-b1^t, 1-b2^t}, Adam's bias corrections for this step
 };
 cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s);
 
 // copies with pitch / dtype / rounding conversion: dst[r][c] = cvt(src[r][c])
 cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt,
                           int64_t ld_src, int rows, int cols, int round, cudaStream_t s);
+// the same copy plus an int32 vector copy (class indices) in one launch; when t is not null the
+// launch also advances the step counter: t += 1, bc = {1 - beta1^t, 1 - beta2^t}
+cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
+                                int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
+                                unsigned long long* t, float* bc, float beta1, float beta2, cudaStream_t s);
 
 // ---- small device helpers ------------------------------------------------------------------
 __device__ __forceinline__ float round_tf32_rne(float x) {

@@ -129,28 +129,54 @@ softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* _
   finish_loss(bt, partials, counter, loss_out, inv_b, red);
 }
 
-// db[n] = sum_b dZ[b][n]: 32 columns x 8 row lanes per block, fixed summation order.
+// db[n] = sum_b dZ[b][n].  Grid (column strips of 32, row chunks): every block sums its rows with
+// 8 row lanes, writes one partial per column to scratch[chunk][n]; the last block of a strip to
+// finish adds the chunk partials in chunk order (fixed order: bit-reproducible) and resets the
+// strip's arrival counter.
+constexpr int kBiasRowsPerChunk = 128;
 template <typename T>
 __global__ void __launch_bounds__(256)
-bias_grad_kernel(const T* __restrict__ dz, int64_t ld, int batch, int n, float* __restrict__ db) {
+bias_grad_kernel(const T* __restrict__ dz, int64_t ld, int batch, int n, float* __restrict__ db,
+                 float* __restrict__ scratch, unsigned int* __restrict__ counters) {
   __shared__ float part[8][33];
-  const int col = blockIdx.x * 32 + (threadIdx.x & 31);
-  const int rl = threadIdx.x >> 5;
+  __shared__ bool is_last;
+  const int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
+  const int col = blockIdx.x * 32 + lane;
+  const int r0 = blockIdx.y * kBiasRowsPerChunk;
+  const int r1 = (gridDim.y == 1) ? batch : min(batch, r0 + kBiasRowsPerChunk);
   float acc = 0.f;
   if (col < n) {
 #pragma unroll 4
-    for (int b = rl; b < batch; b += 8) {
+    for (int b = r0 + rl; b < r1; b += 8) {
       if constexpr (sizeof(T) == 2) acc += __bfloat162float(dz[(int64_t)b * ld + col]);
       else acc += dz[(int64_t)b * ld + col];
     }
   }
-  part[rl][threadIdx.x & 31] = acc;
+  part[rl][lane] = acc;
   __syncthreads();
-  if (rl == 0 && col < n) {
+  if (rl == 0) {
     float s = 0.f;
 #pragma unroll
-    for (int r = 0; r < 8; ++r) s += part[r][threadIdx.x & 31];
-    db[col] = s;
+    for (int r = 0; r < 8; ++r) s += part[r][lane];
+    if (gridDim.y == 1) {
+      if (col < n) db[col] = s;
+    } else if (col < n) {
+      scratch[(int64_t)blockIdx.y * n + col] = s;
+    }
+  }
+  if (gridDim.y == 1) return;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(counters + blockIdx.x, 1u) == gridDim.y - 1);
+  __syncthreads();
+  if (is_last && rl == 0) {
+    __threadfence();
+    if (col < n) {
+      float s = 0.f;
+      for (unsigned int c = 0; c < gridDim.y; ++c) s += __ldcg(scratch + (int64_t)c * n + col);
+      db[col] = s;
+    }
+    if (lane == 0) counters[blockIdx.x] = 0u;
   }
 }
 
@@ -165,7 +191,8 @@ update_kernel(UpdateArgs u) {
   const float4* __restrict__ g4 = reinterpret_cast<const float4*>(u.g);
   float4* __restrict__ s14 = reinterpret_cast<float4*>(u.s1);
   float4* __restrict__ s24 = reinterpret_cast<float4*>(u.s2);
-  const float inv_bc1 = 1.0f / u.bc1, inv_bc2 = 1.0f / u.bc2;
+  float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
+  if constexpr (OPT == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(u.bc); inv_bc2 = 1.0f / __ldg(u.bc + 1); }
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4;
        i += (int64_t)gridDim.x * blockDim.x) {
     float4 p = p4[i];
@@ -228,6 +255,26 @@ copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt
   }
 }
 
+__global__ void __launch_bounds__(256)
+stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows, int cols,
+                    int round, int32_t* cls_dst, const int32_t* cls_src, unsigned long long* t, float* bc,
+                    float beta1, float beta2) {
+  const int64_t total = (int64_t)rows * cols;
+  const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (tid == 0 && t != nullptr) {           // step counter and Adam bias corrections of this step
+    const unsigned long long step = *t + 1ull;
+    *t = step;
+    bc[0] = (float)(1.0 - pow((double)beta1, (double)step));
+    bc[1] = (float)(1.0 - pow((double)beta2, (double)step));
+  }
+  for (int64_t e = tid; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = e / cols, c = e % cols;
+    const float v = apply_round(load_as_float(src, dt, r * ld_src + c), round);
+    store_from_float(dst, dt, r * ld_dst + c, v);
+  }
+  for (int64_t i = tid; i < rows; i += (int64_t)gridDim.x * blockDim.x) cls_dst[i] = cls_src[i];
+}
+
 int grid_for(int64_t work_items, int threads, int max_blocks) {
   int64_t b = (work_items + threads - 1) / threads;
   if (b < 1) b = 1;
@@ -275,15 +322,22 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
   return cudaGetLastError();
 }
 
-int bias_grad_scratch_floats(int, int) { return 0; }
+// scratch: `partials` holds [chunks][n] floats, `counters` one arrival counter per strip of 32 columns
+// (zero-initialised once; the kernel leaves them at zero).  With partials == nullptr one block per
+// strip walks all rows.
+int bias_grad_partial_floats(int batch, int n) {
+  return ((batch + kBiasRowsPerChunk - 1) / kBiasRowsPerChunk) * n;
+}
+int bias_grad_counters(int n) { return (n + 31) / 32; }
 
 cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, int n, float* db,
-                             float*, cudaStream_t s) {
-  const int grid = (n + 31) / 32;
+                             float* partials, unsigned int* counters, cudaStream_t s) {
+  const int chunks = (batch + kBiasRowsPerChunk - 1) / kBiasRowsPerChunk;
+  dim3 grid((n + 31) / 32, (partials == nullptr || counters == nullptr) ? 1 : chunks);
   if (dz_dt == DT_BF16)
-    bias_grad_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)dz, ld, batch, n, db);
+    bias_grad_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)dz, ld, batch, n, db, partials, counters);
   else
-    bias_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dz, ld, batch, n, db);
+    bias_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dz, ld, batch, n, db, partials, counters);
   return cudaGetLastError();
 }
 
@@ -302,6 +356,15 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
     default: return cudaErrorInvalidValue;
   }
 #undef SEGK_UPD
+  return cudaGetLastError();
+}
+
+cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
+                                int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
+                                unsigned long long* t, float* bc, float beta1, float beta2, cudaStream_t s) {
+  const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
+  stage_inputs_kernel<<<grid, 256, 0, s>>>(dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
+                                           beta1, beta2);
   return cudaGetLastError();
 }
 

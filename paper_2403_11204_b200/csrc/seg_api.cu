@@ -7,12 +7,25 @@
 //       [out][ldw] with ldw = in rounded up to 8 elements (16-byte rows for TMA); padding stays 0.
 //   params_op : the same layout in the operand dtype (bf16, or TF32-rounded fp32).
 //   act[l], l = 1..L : [max_batch][ld_l] stored outputs (bf16 or fp32; final logits fp32).
-//   dz[0], dz[1]     : ping-pong dZ buffers, [max_batch][max ld].
+//   dzbuf[l]         : dZ of layer l, [max_batch][ld_{l+1}] (one per layer: the weight-gradient
+//                      branch reads dZ_l while the main branch already produces dZ_{l-1}).
 //   sil              : [M][N_P] fp32 intermediate labels (Eq. 1).
+//
+// One training step is a three-branch dependency graph.  Main branch: forward products, loss, then
+// the dgrad chain.  Gradient branch: per layer the bias gradient and the weight-gradient product
+// (they need dZ_l only).  Update branch: per layer the optimizer update, which waits for that
+// layer's gradients and for its dgrad (the last reader of the old weights).  The HBM-bound updates
+// thereby run beside the tensor-core products of the layers below.  After one eager run per batch size the step is
+// captured into a CUDA graph and replayed; the caller's x / cls are first copied into
+// fixed staging buffers so that the graph never changes.
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
 
+#include <stdlib.h>
+
+#include <algorithm>
+#include <map>
 #include <new>
 #include <string>
 #include <vector>
@@ -53,7 +66,20 @@ struct seg_handle {
   std::vector<int64_t> ld_act;     // index 0..L
   std::vector<int> act_dtype;      // index 1..L
   void* x_stage = nullptr;
-  void* dz[2] = {nullptr, nullptr};
+  int32_t* cls_stage = nullptr;
+  std::vector<void*> dzbuf;        // index 0..L-1
+  float* loss_slot = nullptr;
+  unsigned long long* step_dev = nullptr;
+  float* bc_dev = nullptr;
+  float* bias_scratch = nullptr;
+  unsigned int* bias_counters = nullptr;
+  cudaStream_t side = nullptr, upd = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_join_upd = nullptr;
+  std::vector<cudaEvent_t> ev_dz;  // ev_dz[l]: dZ_l is complete (main branch)
+  std::vector<cudaEvent_t> ev_wg;  // ev_wg[l]: dW_l and db_l are complete (gradient branch)
+  struct StepGraph { int eager_runs = 0; cudaGraphExec_t exec = nullptr; uint64_t kernels = 0; };
+  std::map<int, StepGraph> graphs; // by batch size
+  bool graphs_enabled = true;
   float* sil = nullptr;
   bool have_labels = false;
   float* loss_partials = nullptr;
@@ -106,7 +132,9 @@ seg_status dev_alloc(seg_handle* h, T** out, size_t count, bool zero) {
 struct Launch {
   seg_handle* h;
   bool on;
-  Launch(seg_handle* hh, int kind) : h(hh), on(hh->profile) {
+  cudaStream_t st;
+  Launch(seg_handle* hh, int kind, cudaStream_t stream = nullptr)
+      : h(hh), on(hh->profile), st(stream ? stream : hh->stream) {
     ++h->launches;
     if (!on) return;
     if (h->ev_used + 2 > h->ev_pool.size()) {
@@ -116,25 +144,25 @@ struct Launch {
         h->ev_pool.push_back(e);
       }
     }
-    cudaEventRecord(h->ev_pool[h->ev_used], h->stream);
+    cudaEventRecord(h->ev_pool[h->ev_used], st);
     h->ev_kind.push_back(kind);
   }
   ~Launch() {
     if (!on) return;
-    cudaEventRecord(h->ev_pool[h->ev_used + 1], h->stream);
+    cudaEventRecord(h->ev_pool[h->ev_used + 1], st);
     h->ev_used += 2;
   }
 };
 
-seg_status run_gemm(seg_handle* h, const GemmDesc& g, int kind) {
-  Launch l(h, kind);
+seg_status run_gemm(seg_handle* h, const GemmDesc& g, int kind, cudaStream_t stream) {
+  Launch l(h, kind, stream);
   if (h->use_tc) {
-    cudaError_t e = launch_gemm_tc(g, h->dev_status, h->stream);
+    cudaError_t e = launch_gemm_tc(g, h->dev_status, stream);
     if (e == cudaSuccess) return SEG_OK;
     if (e != cudaErrorNotSupported) return fail_cuda(h, e, "tensor-core product launch");
     cudaGetLastError();
   }
-  SEG_TRY(h, launch_gemm_simt(g, h->stream), "FFMA product launch");
+  SEG_TRY(h, launch_gemm_simt(g, stream), "FFMA product launch");
   return SEG_OK;
 }
 
@@ -162,11 +190,8 @@ seg_status prepare_input(seg_handle* h, const void* x, int batch, const void** x
   return SEG_OK;
 }
 
-seg_status forward_impl(seg_handle* h, const void* x, int batch, const void** x_use, int64_t* ld_x) {
-  const void* a_prev; int64_t ld_prev;
-  seg_status st = prepare_input(h, x, batch, &a_prev, &ld_prev);
-  if (st != SEG_OK) return st;
-  *x_use = a_prev; *ld_x = ld_prev;
+// Forward products of all layers, reading layer 0's input from (a_prev, ld_prev).
+seg_status forward_layers(seg_handle* h, const void* a_prev, int64_t ld_prev, int batch) {
   for (int l = 0; l < h->n_layers; ++l) {
     const LayerInfo& L = h->layers[l];
     const bool last = (l == h->n_layers - 1);
@@ -178,12 +203,19 @@ seg_status forward_impl(seg_handle* h, const void* x, int batch, const void** x_
     g.c_round = (last && h->is_final) ? RND_NONE : h->act_round;
     g.epi = EPI_BIAS_ACT; g.relu = (!last || h->last_relu) ? 1 : 0;
     g.bias = h->params + L.b_off;
-    st = run_gemm(h, g, K_FWD);
+    seg_status st = run_gemm(h, g, K_FWD, h->stream);
     if (st != SEG_OK) return st;
     a_prev = h->act[l + 1]; ld_prev = h->ld_act[l + 1];
   }
   h->last_batch = batch;
   return SEG_OK;
+}
+
+seg_status forward_impl(seg_handle* h, const void* x, int batch) {
+  const void* a_prev; int64_t ld_prev;
+  seg_status st = prepare_input(h, x, batch, &a_prev, &ld_prev);
+  if (st != SEG_OK) return st;
+  return forward_layers(h, a_prev, ld_prev, batch);
 }
 
 seg_status copy_out(seg_handle* h, void* y, int batch) {
@@ -292,10 +324,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   h->act.assign(h->n_layers + 1, nullptr);
   h->ld_act.assign(h->n_layers + 1, 0);
   h->act_dtype.assign(h->n_layers + 1, h->act_dt);
-  int64_t max_ld = 0;
   for (int l = 0; l <= h->n_layers; ++l) {
     h->ld_act[l] = round_up(h->widths[l], 8);
-    if (l >= 1 && h->ld_act[l] > max_ld) max_ld = h->ld_act[l];
   }
   if (h->is_final) h->act_dtype[h->n_layers] = DT_F32;
   for (int l = 1; l <= h->n_layers; ++l) {
@@ -309,11 +339,38 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
     if ((st = dev_alloc(h, &p, (size_t)h->max_batch * h->ld_act[0] * elem_size(h->act_dt), true)) != SEG_OK) return bail(st);
     h->x_stage = p;
   }
-  for (int i = 0; i < 2; ++i) {
-    if (i == 1 && h->n_layers == 1) break;
+  h->dzbuf.assign(h->n_layers, nullptr);
+  for (int l = 0; l < h->n_layers; ++l) {
     char* p = nullptr;
-    if ((st = dev_alloc(h, &p, (size_t)h->max_batch * max_ld * elem_size(h->act_dt), true)) != SEG_OK) return bail(st);
-    h->dz[i] = p;
+    if ((st = dev_alloc(h, &p, (size_t)h->max_batch * h->ld_act[l + 1] * elem_size(h->act_dt), true)) != SEG_OK) return bail(st);
+    h->dzbuf[l] = p;
+  }
+  if ((st = dev_alloc(h, &h->cls_stage, h->max_batch, true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->loss_slot, 1, true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->step_dev, 1, true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->bc_dev, 2, true)) != SEG_OK) return bail(st);
+  {
+    int floats = 0, counters = 0;
+    for (int l = 0; l < h->n_layers; ++l) {
+      floats = std::max(floats, bias_grad_partial_floats(h->max_batch, h->widths[l + 1]));
+      counters = std::max(counters, bias_grad_counters(h->widths[l + 1]));
+    }
+    if ((st = dev_alloc(h, &h->bias_scratch, floats, true)) != SEG_OK) return bail(st);
+    if ((st = dev_alloc(h, &h->bias_counters, counters, true)) != SEG_OK) return bail(st);
+  }
+  if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&h->upd, cudaStreamNonBlocking) != cudaSuccess) return bail(SEG_ERR_CUDA);
+  if (cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_join_upd, cudaEventDisableTiming) != cudaSuccess) return bail(SEG_ERR_CUDA);
+  h->ev_dz.assign(h->n_layers, nullptr);
+  h->ev_wg.assign(h->n_layers, nullptr);
+  for (int l = 0; l < h->n_layers; ++l)
+    if (cudaEventCreateWithFlags(&h->ev_dz[l], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_wg[l], cudaEventDisableTiming) != cudaSuccess) return bail(SEG_ERR_CUDA);
+  {
+    const char* env = getenv("SEG_NO_GRAPH");
+    if (env && env[0] == '1') h->graphs_enabled = false;
   }
   if (!h->is_final &&
       (st = dev_alloc(h, &h->sil, (size_t)h->n_classes * h->widths[h->n_layers], true)) != SEG_OK) return bail(st);
@@ -341,6 +398,16 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
 seg_status seg_destroy(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
   cudaStreamSynchronize(h->stream);
+  if (h->side) cudaStreamSynchronize(h->side);
+  if (h->upd) cudaStreamSynchronize(h->upd);
+  for (auto& kv : h->graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+  for (cudaEvent_t e : h->ev_dz) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_wg) if (e) cudaEventDestroy(e);
+  if (h->ev_join_upd) cudaEventDestroy(h->ev_join_upd);
+  if (h->upd) cudaStreamDestroy(h->upd);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
+  if (h->side) cudaStreamDestroy(h->side);
   for (void* p : h->allocations) cudaFree(p);
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->ev_start) cudaEventDestroy(h->ev_start);
@@ -364,10 +431,93 @@ seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, float kapp
 seg_status seg_forward(seg_handle* h, const void* x, int32_t batch, void* y) {
   if (!h || !x || !y) return SEG_ERR_INVALID_ARG;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
-  const void* x_use; int64_t ld_x;
-  seg_status st = forward_impl(h, x, batch, &x_use, &ld_x);
+  seg_status st = forward_impl(h, x, batch);
   if (st != SEG_OK) return st;
   return copy_out(h, y, batch);
+}
+
+// Enqueues one whole step (forward, loss, backward, update) that reads the staged inputs.
+// forked = false puts all three branches on the main stream (used while profiling).
+static seg_status enqueue_step(seg_handle* h, int batch, bool forked) {
+  const int L = h->n_layers;
+  cudaStream_t mainst = h->stream;
+  cudaStream_t side = forked ? h->side : mainst;
+  cudaStream_t upd = forked ? h->upd : mainst;
+  seg_status st;
+  if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
+  {
+    Launch l(h, K_LOSS, mainst);
+    void* dz_L = h->dzbuf[L - 1];
+    if (h->is_final) {
+      SEG_TRY(h, launch_softmax_ce_loss((const float*)h->act[L], h->ld_act[L], h->cls_stage, h->n_classes, batch,
+                                        h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
+                                        h->loss_partials, h->loss_counter, h->loss_slot, mainst), "softmax-CE loss");
+    } else {
+      SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], h->cls_stage, h->sil, h->widths[L], batch,
+                                 h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
+                                 h->loss_partials, h->loss_counter, h->loss_slot, mainst), "MSE loss");
+    }
+  }
+  if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[L - 1], mainst), "event record");
+  for (int l = L - 1; l >= 0; --l) {
+    const LayerInfo& Ly = h->layers[l];
+    const int64_t ld_dz = h->ld_act[l + 1];
+    const void* dz_l = h->dzbuf[l];
+    const void* a_prev = (l == 0) ? h->x_stage : h->act[l];
+    const int64_t ld_prev = h->ld_act[l];
+    // gradient branch: bias gradient and weight gradient of layer l (need dZ_l)
+    if (forked) SEG_TRY(h, cudaStreamWaitEvent(side, h->ev_dz[l], 0), "stream wait");
+    {
+      Launch lb(h, K_BIAS, side);
+      SEG_TRY(h, launch_bias_grad(dz_l, h->act_dt, ld_dz, batch, Ly.out, h->grads + Ly.b_off, h->bias_scratch, h->bias_counters,
+                                  side),
+              "bias gradient");
+    }
+    GemmDesc w{};
+    w.A = dz_l; w.a_sm = 1; w.a_sk = ld_dz; w.a_dt = h->act_dt;
+    w.B = a_prev; w.b_sk = ld_prev; w.b_sn = 1; w.b_dt = h->act_dt;
+    w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
+    w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
+    if ((st = run_gemm(h, w, K_WGRAD, side)) != SEG_OK) return st;
+    if (forked) SEG_TRY(h, cudaEventRecord(h->ev_wg[l], side), "event record");
+    // main branch: dgrad of layer l, the last reader of the old W_l
+    if (l > 0) {
+      GemmDesc d{};
+      d.A = dz_l; d.a_sm = ld_dz; d.a_sk = 1; d.a_dt = h->act_dt;
+      d.B = weights_op(h, l); d.b_sk = Ly.ldw; d.b_sn = 1; d.b_dt = h->op_dt;
+      d.C = h->dzbuf[l - 1]; d.ldc = h->ld_act[l]; d.c_dt = h->act_dt; d.c_round = h->act_round;
+      d.M = batch; d.N = Ly.in; d.K = Ly.out; d.epi = EPI_MASK;
+      d.mask = h->act[l]; d.ldmask = h->ld_act[l];
+      if ((st = run_gemm(h, d, K_DGRAD, mainst)) != SEG_OK) return st;
+      if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[l - 1], mainst), "event record");
+    }
+    // update branch: layer l's tensors (W_l and b_l are adjacent in the flat range)
+    if (forked) {
+      SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_wg[l], 0), "stream wait");
+      if (l > 0) SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_dz[l - 1], 0), "stream wait");   // dgrad(l) done
+    }
+    const int64_t lo = Ly.w_off;
+    const int64_t hi = (l + 1 < L) ? h->layers[l + 1].w_off : h->n_flat;
+    UpdateArgs u{};
+    u.p = h->params + lo; u.g = h->grads + lo;
+    u.s1 = h->state1 ? h->state1 + lo : nullptr; u.s2 = h->state2 ? h->state2 + lo : nullptr;
+    u.p_op = h->params_op ? (void*)(reinterpret_cast<char*>(h->params_op) + lo * elem_size(h->op_dt)) : nullptr;
+    u.op_dt = h->op_dt; u.op_round = h->op_round;
+    u.n = hi - lo; u.optimizer = h->optimizer;
+    u.lr = h->lr; u.momentum = h->momentum; u.beta1 = h->beta1; u.beta2 = h->beta2; u.eps = h->eps;
+    u.bc = h->bc_dev;
+    {
+      Launch lu(h, K_UPDATE, upd);
+      SEG_TRY(h, launch_update(u, upd), "optimizer update");
+    }
+  }
+  if (forked) {
+    SEG_TRY(h, cudaEventRecord(h->ev_join, side), "event record");
+    SEG_TRY(h, cudaEventRecord(h->ev_join_upd, upd), "event record");
+    SEG_TRY(h, cudaStreamWaitEvent(mainst, h->ev_join, 0), "stream wait");
+    SEG_TRY(h, cudaStreamWaitEvent(mainst, h->ev_join_upd, 0), "stream wait");
+  }
+  return SEG_OK;
 }
 
 seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
@@ -375,68 +525,56 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
   if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   if (!h->is_final && !h->have_labels) return SEG_ERR_STATE;
-  const int L = h->n_layers;
-  const void* x_use; int64_t ld_x;   // where layer 0 read its input (the caller's x or the staged copy)
-  seg_status st = forward_impl(h, x, batch, &x_use, &ld_x);
-  if (st != SEG_OK) return st;
-  if (y_out && (st = copy_out(h, y_out, batch)) != SEG_OK) return st;
-
-  // loss -> dZ_L
-  void* dz_cur = h->dz[(L - 1) & 1];
+  seg_status st = SEG_OK;
   {
-    Launch l(h, K_LOSS);
-    if (h->is_final) {
-      SEG_TRY(h, launch_softmax_ce_loss((const float*)h->act[L], h->ld_act[L], cls, h->n_classes, batch,
-                                        h->last_relu ? 1 : 0, dz_cur, h->act_dt, h->act_round, h->ld_act[L],
-                                        h->loss_partials, h->loss_counter, loss_out, h->stream), "softmax-CE loss");
+    // fixed staging buffers: rounds x in TF32 mode, pads the pitch, keeps the graph's pointers constant;
+    // the same launch advances the device-side step counter and Adam's bias corrections
+    Launch lc(h, K_COPY);
+    SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
+                                   h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
+                                   h->stream), "input staging");
+  }
+  if (h->profile || !h->graphs_enabled) {
+    st = enqueue_step(h, batch, !h->profile);
+  } else {
+    seg_handle::StepGraph& g = h->graphs[batch];
+    if (g.exec != nullptr) {
+      SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
+      h->launches += g.kernels;
+    } else if (g.eager_runs == 0) {
+      st = enqueue_step(h, batch, true);      // first step at this batch size: eager (also sets kernel attributes)
+      g.eager_runs = 1;
     } else {
-      SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], cls, h->sil, h->widths[L], batch,
-                                 h->last_relu ? 1 : 0, dz_cur, h->act_dt, h->act_round, h->ld_act[L],
-                                 h->loss_partials, h->loss_counter, loss_out, h->stream), "MSE loss");
+      const uint64_t before = h->launches;
+      cudaGraph_t graph = nullptr;
+      if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        h->graphs_enabled = false;
+        st = enqueue_step(h, batch, true);
+      } else {
+        st = enqueue_step(h, batch, true);
+        cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
+        if (st == SEG_OK && e == cudaSuccess && graph != nullptr &&
+            cudaGraphInstantiate(&g.exec, graph, 0) == cudaSuccess) {
+          g.kernels = h->launches - before;
+          SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
+        } else {
+          // capture did not work here: run eagerly from now on
+          cudaGetLastError();
+          g.exec = nullptr;
+          h->graphs_enabled = false;
+          h->launches = before;
+          st = enqueue_step(h, batch, true);
+        }
+        if (graph) cudaGraphDestroy(graph);
+      }
     }
   }
-  // backward, layer by layer; dgrad of layer l is issued before anything overwrites W_l
-  for (int l = L - 1; l >= 0; --l) {
-    const LayerInfo& Ly = h->layers[l];
-    const int64_t ld_dz = h->ld_act[l + 1];
-    const void* a_prev = (l == 0) ? x_use : h->act[l];
-    const int64_t ld_prev = (l == 0) ? ld_x : h->ld_act[l];
-    {
-      Launch lb(h, K_BIAS);
-      SEG_TRY(h, launch_bias_grad(dz_cur, h->act_dt, ld_dz, batch, Ly.out, h->grads + Ly.b_off, nullptr,
-                                  h->stream), "bias gradient");
-    }
-    GemmDesc w{};
-    w.A = dz_cur; w.a_sm = 1; w.a_sk = ld_dz; w.a_dt = h->act_dt;
-    w.B = a_prev; w.b_sk = ld_prev; w.b_sn = 1; w.b_dt = h->act_dt;
-    w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
-    w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
-    if ((st = run_gemm(h, w, K_WGRAD)) != SEG_OK) return st;
-    if (l > 0) {
-      void* dz_next = h->dz[(l - 1) & 1];
-      GemmDesc d{};
-      d.A = dz_cur; d.a_sm = ld_dz; d.a_sk = 1; d.a_dt = h->act_dt;
-      d.B = weights_op(h, l); d.b_sk = Ly.ldw; d.b_sn = 1; d.b_dt = h->op_dt;
-      d.C = dz_next; d.ldc = h->ld_act[l]; d.c_dt = h->act_dt; d.c_round = h->act_round;
-      d.M = batch; d.N = Ly.in; d.K = Ly.out; d.epi = EPI_MASK;
-      d.mask = h->act[l]; d.ldmask = h->ld_act[l];
-      if ((st = run_gemm(h, d, K_DGRAD)) != SEG_OK) return st;
-      dz_cur = dz_next;
-    }
-  }
-  // optimizer
+  if (st != SEG_OK) return st;
   ++h->step;
-  UpdateArgs u{};
-  u.p = h->params; u.g = h->grads; u.s1 = h->state1; u.s2 = h->state2;
-  u.p_op = h->params_op; u.op_dt = h->op_dt; u.op_round = h->op_round;
-  u.n = h->n_flat; u.optimizer = h->optimizer;
-  u.lr = h->lr; u.momentum = h->momentum; u.beta1 = h->beta1; u.beta2 = h->beta2; u.eps = h->eps;
-  u.bc1 = (float)(1.0 - pow((double)h->beta1, (double)h->step));
-  u.bc2 = (float)(1.0 - pow((double)h->beta2, (double)h->step));
-  {
-    Launch lu(h, K_UPDATE);
-    SEG_TRY(h, launch_update(u, h->stream), "optimizer update");
-  }
+  if (loss_out)
+    SEG_TRY(h, cudaMemcpyAsync(loss_out, h->loss_slot, sizeof(float), cudaMemcpyDeviceToDevice, h->stream), "loss copy");
+  if (y_out && (st = copy_out(h, y_out, batch)) != SEG_OK) return st;
   return SEG_OK;
 }
 
@@ -530,6 +668,9 @@ seg_status seg_get_step(const seg_handle* h, uint64_t* step) {
 seg_status seg_set_step(seg_handle* h, uint64_t step) {
   if (!h) return SEG_ERR_INVALID_ARG;
   h->step = step;
+  const unsigned long long t = step;
+  SEG_TRY(h, cudaMemcpyAsync(h->step_dev, &t, sizeof(t), cudaMemcpyHostToDevice, h->stream), "step counter copy");
+  SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
   return SEG_OK;
 }
 
