@@ -18,10 +18,18 @@
 // 8-row groups 1024 bytes apart); 32-bit MN-major tiles must use the 128-byte swizzle with
 // 32-byte atoms (4-row groups 512 bytes apart), in the tensor map and in the descriptor alike.
 //
+// Small problems (few output tiles, long K) use gemm_tc_splitk_kernel instead: a thread-block
+// cluster of 2, 4 or 8 CTAs shares one 128 x 64 output tile, each CTA contracts its own slice of K
+// into TMEM, and the partial tiles are combined through distributed shared memory as a
+// reduce-scatter (every CTA bulk-copies column slice j of its partial into CTA j's shared memory;
+// CTA j adds what it received and runs the epilogue on that slice).  One SM's shared-memory fill rate bounds a single CTA's main loop, so spreading K over a
+// cluster shortens exactly the part of the kernel that grows with the problem.
+//
 // Every wait on an mbarrier is bounded: after about two seconds the waiting thread raises an abort
 // flag, records DEV_TIMEOUT in the status word and all roles leave their loops; TMEM is released
 // before the CTA exits.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -162,20 +170,27 @@ struct SmemLayout {
   static constexpr int TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
 };
 
-// Epilogue for 32 consecutive columns of one row.
+// Epilogue for up to 32 consecutive columns of one row.  Columns are handled in groups of 8 with
+// 16-byte accesses when the group count is whole and the row segment is 16-byte aligned (every
+// lane touches its own row, so wide accesses are what keeps the number of memory wavefronts down);
+// ragged or unaligned segments fall back to scalar accesses.
 __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], int row, int col0,
                                                int n_total) {
   const int n_valid = min(32, n_total - col0);
+  const bool whole = (n_valid & 7) == 0;
   if (e.epi == EPI_BIAS_ACT) {
-    if (n_valid == 32) {
+    const float* brow = e.bias + col0;
+    if (whole && ((reinterpret_cast<uintptr_t>(brow) & 15u) == 0)) {
 #pragma unroll
       for (int j = 0; j < 32; j += 4) {
-        const float4 b = __ldg(reinterpret_cast<const float4*>(e.bias + col0 + j));
-        v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+        if (j < n_valid) {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(brow + j));
+          v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+        }
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __ldg(e.bias + col0 + j);
+      for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __ldg(brow + j);
     }
     if (e.relu) {
 #pragma unroll
@@ -184,17 +199,19 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
   } else if (e.epi == EPI_MASK) {
     if (e.c_dt == DT_BF16) {
       const __nv_bfloat16* mrow = reinterpret_cast<const __nv_bfloat16*>(e.mask) + (int64_t)row * e.ldmask + col0;
-      if (n_valid == 32) {
+      if (whole && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0)) {
 #pragma unroll
         for (int j = 0; j < 32; j += 8) {
-          const uint4 q = __ldg(reinterpret_cast<const uint4*>(mrow + j));
-          const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+          if (j < n_valid) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(mrow + j));
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            // a bf16 is positive iff its sign bit is clear and it is not zero
-            const uint32_t lo = w[t] & 0xFFFFu, hi = w[t] >> 16;
-            if (!(lo != 0u && lo < 0x8000u)) v[j + 2 * t] = 0.f;
-            if (!(hi != 0u && hi < 0x8000u)) v[j + 2 * t + 1] = 0.f;
+            for (int t = 0; t < 4; ++t) {
+              // a bf16 is positive iff its sign bit is clear and it is not zero
+              const uint32_t lo = w[t] & 0xFFFFu, hi = w[t] >> 16;
+              if (!(lo != 0u && lo < 0x8000u)) v[j + 2 * t] = 0.f;
+              if (!(hi != 0u && hi < 0x8000u)) v[j + 2 * t + 1] = 0.f;
+            }
           }
         }
       } else {
@@ -204,9 +221,22 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
       }
     } else {
       const float* mrow = reinterpret_cast<const float*>(e.mask) + (int64_t)row * e.ldmask + col0;
+      if (whole && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0)) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (j < n_valid && !(__ldg(mrow + j) > 0.f)) v[j] = 0.f;
+        for (int j = 0; j < 32; j += 4) {
+          if (j < n_valid) {
+            const float4 m = __ldg(reinterpret_cast<const float4*>(mrow + j));
+            if (!(m.x > 0.f)) v[j] = 0.f;
+            if (!(m.y > 0.f)) v[j + 1] = 0.f;
+            if (!(m.z > 0.f)) v[j + 2] = 0.f;
+            if (!(m.w > 0.f)) v[j + 3] = 0.f;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (j < n_valid && !(__ldg(mrow + j) > 0.f)) v[j] = 0.f;
+      }
     }
   }
   if (e.c_round == RND_TF32) {
@@ -215,17 +245,19 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
   }
   if (e.c_dt == DT_BF16) {
     __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(e.C) + (int64_t)row * e.ldc + col0;
-    if (n_valid == 32 && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
+    if (whole && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
 #pragma unroll
       for (int j = 0; j < 32; j += 8) {
-        uint4 q;
-        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]);
-        __nv_bfloat162 p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
-        __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
-        __nv_bfloat162 p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
-        q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
-        q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
-        *reinterpret_cast<uint4*>(crow + j) = q;
+        if (j < n_valid) {
+          uint4 q;
+          __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]);
+          __nv_bfloat162 p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+          __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
+          __nv_bfloat162 p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+          q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
+          q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
+          *reinterpret_cast<uint4*>(crow + j) = q;
+        }
       }
     } else {
 #pragma unroll
@@ -233,10 +265,11 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
     }
   } else {
     float* crow = reinterpret_cast<float*>(e.C) + (int64_t)row * e.ldc + col0;
-    if (n_valid == 32 && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
+    if (whole && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 4)
-        *reinterpret_cast<float4*>(crow + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      for (int j = 0; j < 32; j += 4) {
+        if (j < n_valid) *reinterpret_cast<float4*>(crow + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      }
     } else {
 #pragma unroll
       for (int j = 0; j < 32; ++j) if (j < n_valid) crow[j] = v[j];
@@ -398,6 +431,216 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+
+// ---- cluster helpers (split-K kernel) -----------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank)); return r;
+}
+// bulk copy from this CTA's shared memory into a peer's; completes (by bytes) on the peer's mbarrier
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster_addr, uint32_t src_local_addr,
+                                                  uint32_t bytes, uint32_t bar_cluster_addr) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster_addr), "r"(src_local_addr), "r"(bytes), "r"(bar_cluster_addr) : "memory");
+}
+constexpr int SPLITK_BLOCK_N = 64;
+constexpr int SPLITK_STAGES = 6;
+constexpr int SPLITK_STAGE_BYTES = A_TILE_BYTES + SPLITK_BLOCK_N * TILE_ROW_BYTES;       // 24 KiB
+constexpr int SPLITK_RECV_BYTES = 8 * (SPLITK_BLOCK_N / 8) * BLOCK_M * 4;                // [src][col in slice][row] fp32, 32 KiB
+constexpr int SPLITK_SMEM = SPLITK_STAGES * SPLITK_STAGE_BYTES + 2 * SPLITK_RECV_BYTES + SMEM_EXTRA;   // + send buffer
+
+// One 128 x 64 output tile per cluster; CTA r of the cluster contracts k-blocks [r*kpc, (r+1)*kpc).
+template <bool TF32, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                      int M, int N, int K, int split, EpilogueArgs epi, int* dev_status) {
+  constexpr int BLOCK_N = SPLITK_BLOCK_N;
+  constexpr int STAGES = SPLITK_STAGES;
+  constexpr int B_TILE_BYTES = BLOCK_N * TILE_ROW_BYTES;
+  constexpr int BLOCK_K = TF32 ? 32 : 64;
+  constexpr int UMMA_K = TF32 ? 8 : 16;
+  constexpr int CHUNK = TF32 ? 32 : 64;
+  constexpr int MN_CHUNK_BYTES = BLOCK_K * TILE_ROW_BYTES;
+  constexpr uint32_t TMEM_COLS = BLOCK_N;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * A_TILE_BYTES;
+  float* recv = reinterpret_cast<float*>(smem + STAGES * SPLITK_STAGE_BYTES);                      // [src][col in slice][row]
+  float* send = reinterpret_cast<float*>(smem + STAGES * SPLITK_STAGE_BYTES + SPLITK_RECV_BYTES);  // [dest][col in slice][row]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * SPLITK_STAGE_BYTES + 2 * SPLITK_RECV_BYTES);
+  // bars[0..S) full, [S..2S) empty, [2S] accumulator complete, [2S+1] partial slices received
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  const uint32_t acc_bar = bar_base + 8u * (2 * STAGES);
+  const uint32_t recv_bar = bar_base + 8u * (2 * STAGES + 1);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_bar, 1);
+    mbar_init(recv_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // this CTA will receive one column slice (BLOCK_N / split columns x 128 rows, fp32) from every peer
+    mbar_arrive_expect_tx(recv_bar, (uint32_t)((split - 1) * (BLOCK_N / split) * BLOCK_M * 4));
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();                   // "my barriers are initialised"; the matching wait sits in front of the
+  tc_fence_after();                   // first remote access (the slice exchange), off the main loop's path
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
+  const int tile = blockIdx.x / split;
+  const int m0 = (tile % tiles_m) * BLOCK_M, n0 = (tile / tiles_m) * BLOCK_N;
+  const int num_k = (K + BLOCK_K - 1) / BLOCK_K;
+  const int kpc = (num_k + split - 1) / split;
+  const int kb_begin = min(num_k, (int)rank * kpc), kb_end = min(num_k, kb_begin + kpc);
+  const int my_k = kb_end - kb_begin;     // may be 0 for the last ranks: they contribute zeros
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) break;
+        mbar_arrive_expect_tx(full_bar(stage), (uint32_t)SPLITK_STAGE_BYTES);
+        const uint32_t a_dst = smem_u32(smem_a + stage * A_TILE_BYTES);
+        const uint32_t b_dst = smem_u32(smem_b + stage * B_TILE_BYTES);
+        const int k0 = kb * BLOCK_K;
+        if constexpr (A_MN) {
+#pragma unroll
+          for (int c = 0; c < BLOCK_M / CHUNK; ++c)
+            tma_load_2d(a_dst + c * MN_CHUNK_BYTES, &map_a, m0 + c * CHUNK, k0, full_bar(stage));
+        } else {
+          tma_load_2d(a_dst, &map_a, k0, m0, full_bar(stage));
+        }
+        if constexpr (B_MN) {
+#pragma unroll
+          for (int c = 0; c < BLOCK_N / CHUNK; ++c)
+            tma_load_2d(b_dst + c * MN_CHUNK_BYTES, &map_b, n0 + c * CHUNK, k0, full_bar(stage));
+        } else {
+          tma_load_2d(b_dst, &map_b, k0, n0, full_bar(stage));
+        }
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t fmt = TF32 ? 2u : 1u;
+      constexpr uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BLOCK_N >> 3) << 17) |
+                                 ((uint32_t)(BLOCK_M >> 4) << 24);
+      constexpr uint32_t a_lbo = A_MN ? MN_CHUNK_BYTES : 16, b_lbo = B_MN ? MN_CHUNK_BYTES : 16;
+      constexpr uint32_t a_kstep = A_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      constexpr uint32_t b_kstep = B_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      constexpr uint32_t a_sbo = (TF32 && A_MN) ? 512 : 1024, b_sbo = (TF32 && B_MN) ? 512 : 1024;
+      constexpr uint32_t a_lay = (TF32 && A_MN) ? 1 : 2, b_lay = (TF32 && B_MN) ? 1 : 2;
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = 0; kb < my_k; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase, abort_flag, dev_status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_src = smem_u32(smem_a + stage * A_TILE_BYTES);
+        const uint32_t b_src = smem_u32(smem_b + stage * B_TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
+          const uint64_t da = make_smem_desc(a_src + kk * a_kstep, a_lbo, a_sbo, a_lay);
+          const uint64_t db = make_smem_desc(b_src + kk * b_kstep, b_lbo, b_sbo, b_lay);
+          tc_mma<TF32>(tmem_base, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(empty_bar(stage));
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (ok) {
+        if (my_k > 0) tc_commit(acc_bar);
+        else mbar_arrive(acc_bar);          // nothing to contract: the epilogue treats the partial as zero
+      }
+    }
+  } else {
+    // ---------------- epilogue warps: reduce-scatter across the cluster, then the usual epilogue ------------
+    const int quarter = warp & 3;
+    const int row_in_tile = quarter * 32 + lane;
+    const int row = m0 + row_in_tile;
+    const int w = BLOCK_N / split;                         // columns owned by each CTA: 32, 16 or 8
+    bool ok = mbar_wait(acc_bar, 0, abort_flag, dev_status);
+    tc_fence_after();
+    const uint32_t slice_bytes = (uint32_t)(w * BLOCK_M * 4);
+    float own[32];                                         // this CTA's slice of its own partial (w <= 32 used)
+#pragma unroll
+    for (int j = 0; j < 32; ++j) own[j] = 0.f;
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < BLOCK_N / 32; ++c) {
+        float v[32];
+        if (my_k > 0) {
+          tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0.f;
+        }
+        // column c*32+j belongs to CTA (c*32+j)/w; the send buffer is [dest][col in slice][row], which is
+        // simply [column][row]: consecutive lanes write consecutive floats
+#pragma unroll
+        for (int j = 0; j < 32; ++j) send[(c * 32 + j) * BLOCK_M + row_in_tile] = v[j];
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk copies
+      cluster_wait();                                                // every peer's receive barrier exists
+      asm volatile("bar.sync 1, 128;" ::: "memory");                 // the four epilogue warps
+      if (warp == 2 && lane == 0) {
+        for (uint32_t dest = 0; dest < (uint32_t)split; ++dest) {
+          if (dest == rank) continue;
+          const uint32_t src = smem_u32(send + (int)dest * w * BLOCK_M);
+          const uint32_t dst = map_to_cta(smem_u32(recv + (int)rank * w * BLOCK_M), dest);
+          bulk_copy_to_peer(dst, src, slice_bytes, map_to_cta(recv_bar, dest));
+        }
+      }
+      ok = mbar_wait(recv_bar, 0, abort_flag, dev_status);
+    } else {
+      cluster_wait();
+    }
+    if (ok) {
+#pragma unroll
+      for (int cs = 0; cs < 32; ++cs)
+        if (cs < w) own[cs] = send[((int)rank * w + cs) * BLOCK_M + row_in_tile];
+      for (int src = 0; src < split; ++src) {
+        if ((uint32_t)src == rank) continue;
+#pragma unroll
+        for (int cs = 0; cs < 32; ++cs)
+          if (cs < w) own[cs] += recv[(src * w + cs) * BLOCK_M + row_in_tile];
+      }
+      const int col0 = n0 + (int)rank * w;
+      if (row < M && col0 < N) epilogue_store(epi, own, row, col0, min(N, col0 + w));
+    }
+    tc_fence_before();
+  }
+
+  __syncwarp();
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  }
+  if (warp < 2) cluster_wait();       // the producer and MMA warps complete the first cluster phase here
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();                   // no CTA leaves while a peer may still read its send buffer or write
+  cluster_wait();                     // into its receive buffer
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -406,6 +649,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
 bool g_init_done = false, g_init_ok = false;
+bool g_allow_splitk = true;
 
 // 2-D tensor map over a row-major matrix: `inner` contiguous elements per row, `outer` rows,
 // `row_stride_bytes` between rows; box = box_inner x box_outer; 128-byte swizzle (32-byte atoms
@@ -450,6 +694,55 @@ cudaError_t launch_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUt
   return cudaErrorNotSupported;
 }
 
+
+template <bool TF32, bool A_MN, bool B_MN>
+cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
+                                  const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
+  auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SPLITK_SMEM);
+    if (err != cudaSuccess) return err;
+    attr_set = true;
+  }
+  const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + SPLITK_BLOCK_N - 1) / SPLITK_BLOCK_N);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SPLITK_SMEM;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, g.M, g.N, g.K, split, e, dev_status);
+}
+
+template <bool TF32>
+cudaError_t launch_splitk_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUtensorMap& mb,
+                                 const GemmDesc& g, const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
+  if (!a_mn && !b_mn) return launch_splitk_variant<TF32, false, false>(ma, mb, g, e, split, dev_status, s);
+  if (!a_mn && b_mn) return launch_splitk_variant<TF32, false, true>(ma, mb, g, e, split, dev_status, s);
+  if (a_mn && b_mn) return launch_splitk_variant<TF32, true, true>(ma, mb, g, e, split, dev_status, s);
+  return cudaErrorNotSupported;
+}
+
+// Split K over a cluster when the 128 x 64 tiles alone would leave most SMs idle and K is long
+// enough that the main loop, not the fixed cost, dominates.  Returns 1 for "do not split".
+int pick_split(int M, int N, int K, bool tf32) {
+  const int tiles = ((M + BLOCK_M - 1) / BLOCK_M) * ((N + SPLITK_BLOCK_N - 1) / SPLITK_BLOCK_N);
+  const int num_k = (K + (tf32 ? 32 : 64) - 1) / (tf32 ? 32 : 64);
+  // measured: a k-block costs about 0.27 us of one SM's shared-memory fill time, the cluster exchange about 2 us
+  int best = 1;
+  double best_us = 0.27 * num_k;
+  for (int sp : {2, 4}) {
+    if (tiles * sp > g_num_sms) break;
+    const double us = 0.27 * ((num_k + sp - 1) / sp) + 2.0;
+    if (us < best_us - 0.5) { best = sp; best_us = us; }
+  }
+  return best;
+}
+
 int pick_block_n(int M, int N) {
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   int best = 64; long best_cost = -1;
@@ -479,6 +772,8 @@ bool gemm_tc_init() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
   if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  const char* env = getenv("SEG_NO_SPLITK");
+  if (env && env[0] == '1') g_allow_splitk = false;
   g_init_ok = g_num_sms > 0;
   return g_init_ok;
 }
@@ -504,7 +799,8 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   if ((a_pitch * esz) % 16 != 0 || (b_pitch * esz) % 16 != 0) return cudaErrorNotSupported;
   if (a_pitch * (int64_t)esz >= (1ll << 40) || b_pitch * (int64_t)esz >= (1ll << 40)) return cudaErrorNotSupported;
 
-  const int block_n = pick_block_n(g.M, g.N);
+  const int split = g_allow_splitk ? pick_split(g.M, g.N, g.K, tf32) : 1;
+  const int block_n = split > 1 ? SPLITK_BLOCK_N : pick_block_n(g.M, g.N);
   const uint32_t block_k = tf32 ? 32 : 64, chunk = tf32 ? 32 : 64;
   CUtensorMap ma, mb;
   bool ok;
@@ -519,6 +815,10 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   e.C = g.C; e.ldc = g.ldc; e.c_dt = g.c_dt; e.c_round = g.c_round; e.epi = g.epi; e.relu = g.relu;
   e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
 
+  if (split > 1) {
+    return tf32 ? launch_splitk_majors<true>(a_mn, b_mn, ma, mb, g, e, split, dev_status, s)
+                : launch_splitk_majors<false>(a_mn, b_mn, ma, mb, g, e, split, dev_status, s);
+  }
 #define SEGK_TC(TF, BN) launch_majors<TF, BN>(a_mn, b_mn, ma, mb, g, e, dev_status, s)
   if (tf32) {
     if (block_n == 256) return SEGK_TC(true, 256);
