@@ -344,6 +344,18 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
     return out
 
 
+def aggregate_over_ranks(ms_total, steps, batch, world, device="cuda"):
+    """Replicas only: the job's time is the slowest rank's, its work the sum over ranks.
+    Returns (samples/s of the whole job, ms of the timed region)."""
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    return world * steps * batch / (ms_total * 1e-3), ms_total
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -392,10 +404,8 @@ def main():
     res = measure(w, args.steps, args.warmup, peaks, device_index=local_rank, full=True,
                   n_samples=args.samples or None)
     ms_total = res["ms_per_step"] * args.steps
+    value, ms_total = aggregate_over_ranks(ms_total, args.steps, w.batch, world)
     if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
         e = torch.tensor([res["e2e"]["value"]], device="cuda")
         dist.all_reduce(e, op=dist.ReduceOp.SUM)
         res["e2e"]["value"] = float(e.item())
@@ -404,7 +414,6 @@ def main():
         if world > 1:
             dist.destroy_process_group()
         return
-    value = world * args.steps * w.batch / (ms_total * 1e-3)
     line = {"metric": "segment train-step samples/sec", "value": value, "unit": "samples/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

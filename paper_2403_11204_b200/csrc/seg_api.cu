@@ -77,9 +77,23 @@ struct seg_handle {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_join_upd = nullptr;
   std::vector<cudaEvent_t> ev_dz;  // ev_dz[l]: dZ_l is complete (main branch)
   std::vector<cudaEvent_t> ev_wg;  // ev_wg[l]: dW_l and db_l are complete (gradient branch)
-  struct StepGraph { int eager_runs = 0; cudaGraphExec_t exec = nullptr; uint64_t kernels = 0; };
+  // A captured step.  The caller's pointers enter the graph in two kernel nodes only (input staging:
+  // x and cls; loss: loss_out); their parameters are rewritten before every replay.
+  struct StepGraph {
+    int eager_runs = 0;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    uint64_t kernels = 0;
+    cudaGraphNode_t stage_node = nullptr, loss_node = nullptr;
+    cudaKernelNodeParams stage_params{}, loss_params{};
+    std::vector<void*> stage_args, loss_args;
+    const void* cur_x = nullptr; const int32_t* cur_cls = nullptr; float* cur_loss = nullptr;   // now in the exec
+  };
+  cudaGraphNode_t cap_stage_node = nullptr, cap_loss_node = nullptr;   // filled while capturing
+  bool capturing = false;
   std::map<int, StepGraph> graphs; // by batch size
   bool graphs_enabled = true;
+  bool fork_enabled = true;        // run the gradient and update branches on their own streams
   float* sil = nullptr;
   bool have_labels = false;
   float* loss_partials = nullptr;
@@ -371,6 +385,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   {
     const char* env = getenv("SEG_NO_GRAPH");
     if (env && env[0] == '1') h->graphs_enabled = false;
+    env = getenv("SEG_NO_FORK");
+    if (env && env[0] == '1') h->fork_enabled = false;
   }
   if (!h->is_final &&
       (st = dev_alloc(h, &h->sil, (size_t)h->n_classes * h->widths[h->n_layers], true)) != SEG_OK) return bail(st);
@@ -400,7 +416,10 @@ seg_status seg_destroy(seg_handle* h) {
   cudaStreamSynchronize(h->stream);
   if (h->side) cudaStreamSynchronize(h->side);
   if (h->upd) cudaStreamSynchronize(h->upd);
-  for (auto& kv : h->graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+  for (auto& kv : h->graphs) {
+    if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+    if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
+  }
   for (cudaEvent_t e : h->ev_dz) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : h->ev_wg) if (e) cudaEventDestroy(e);
   if (h->ev_join_upd) cudaEventDestroy(h->ev_join_upd);
@@ -438,12 +457,36 @@ seg_status seg_forward(seg_handle* h, const void* x, int32_t batch, void* y) {
 
 // Enqueues one whole step (forward, loss, backward, update) that reads the staged inputs.
 // forked = false puts all three branches on the main stream (used while profiling).
-static seg_status enqueue_step(seg_handle* h, int batch, bool forked) {
+static cudaGraphNode_t last_captured_node(seg_handle* h) {
+  cudaStreamCaptureStatus status;
+  unsigned long long id = 0;
+  cudaGraph_t graph = nullptr;
+  const cudaGraphNode_t* deps = nullptr;
+  size_t n = 0;
+  if (cudaStreamGetCaptureInfo(h->stream, &status, &id, &graph, &deps, &n) != cudaSuccess || n != 1) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return deps[0];
+}
+
+static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void* x, const int32_t* cls,
+                               float* loss_out) {
   const int L = h->n_layers;
   cudaStream_t mainst = h->stream;
   cudaStream_t side = forked ? h->side : mainst;
   cudaStream_t upd = forked ? h->upd : mainst;
   seg_status st;
+  float* loss_dst = loss_out ? loss_out : h->loss_slot;
+  {
+    // fixed staging buffers: rounds x in TF32 mode, pads the pitch, keeps every later pointer constant;
+    // the same launch advances the device-side step counter and Adam's bias corrections
+    Launch lc(h, K_COPY);
+    SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
+                                   h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
+                                   mainst), "input staging");
+  }
+  if (h->capturing) h->cap_stage_node = last_captured_node(h);
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
   {
     Launch l(h, K_LOSS, mainst);
@@ -451,13 +494,14 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked) {
     if (h->is_final) {
       SEG_TRY(h, launch_softmax_ce_loss((const float*)h->act[L], h->ld_act[L], h->cls_stage, h->n_classes, batch,
                                         h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
-                                        h->loss_partials, h->loss_counter, h->loss_slot, mainst), "softmax-CE loss");
+                                        h->loss_partials, h->loss_counter, loss_dst, mainst), "softmax-CE loss");
     } else {
       SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], h->cls_stage, h->sil, h->widths[L], batch,
                                  h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
-                                 h->loss_partials, h->loss_counter, h->loss_slot, mainst), "MSE loss");
+                                 h->loss_partials, h->loss_counter, loss_dst, mainst), "MSE loss");
     }
   }
+  if (h->capturing) h->cap_loss_node = last_captured_node(h);
   if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[L - 1], mainst), "event record");
   for (int l = L - 1; l >= 0; --l) {
     const LayerInfo& Ly = h->layers[l];
@@ -520,29 +564,59 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked) {
   return SEG_OK;
 }
 
+// Index of the caller-supplied pointers in the kernels' parameter lists (see elementwise.cu).
+static const int kStageArgCount = 14, kStageArgX = 3, kStageArgCls = 9;
+static int loss_arg_count(const seg_handle* h) { return h->is_final ? 12 : 13; }
+
+static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGraph_t graph) {
+  if (!h->cap_stage_node || !h->cap_loss_node) return false;
+  g.stage_node = h->cap_stage_node; g.loss_node = h->cap_loss_node;
+  if (cudaGraphKernelNodeGetParams(g.stage_node, &g.stage_params) != cudaSuccess) return false;
+  if (cudaGraphKernelNodeGetParams(g.loss_node, &g.loss_params) != cudaSuccess) return false;
+  g.stage_args.assign(g.stage_params.kernelParams, g.stage_params.kernelParams + kStageArgCount);
+  g.loss_args.assign(g.loss_params.kernelParams, g.loss_params.kernelParams + loss_arg_count(h));
+  if (cudaGraphInstantiate(&g.exec, graph, 0) != cudaSuccess) { g.exec = nullptr; return false; }
+  g.graph = graph;                      // kept alive: the parameter blocks above belong to it
+  return true;
+}
+
+static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const void* x, const int32_t* cls,
+                               float* loss_out) {
+  float* loss_dst = loss_out ? loss_out : h->loss_slot;
+  if (x != g.cur_x || cls != g.cur_cls) {
+    g.stage_args[kStageArgX] = (void*)&x;
+    g.stage_args[kStageArgCls] = (void*)&cls;
+    cudaKernelNodeParams sp = g.stage_params;
+    sp.kernelParams = g.stage_args.data();
+    SEG_TRY(h, cudaGraphExecKernelNodeSetParams(g.exec, g.stage_node, &sp), "graph parameter update");
+    g.cur_x = x; g.cur_cls = cls;
+  }
+  if (loss_dst != g.cur_loss) {
+    g.loss_args[loss_arg_count(h) - 1] = (void*)&loss_dst;
+    cudaKernelNodeParams lp = g.loss_params;
+    lp.kernelParams = g.loss_args.data();
+    SEG_TRY(h, cudaGraphExecKernelNodeSetParams(g.exec, g.loss_node, &lp), "graph parameter update");
+    g.cur_loss = loss_dst;
+  }
+  SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
+  h->launches += g.kernels;
+  return SEG_OK;
+}
+
 seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
                           float* loss_out, void* y_out) {
   if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   if (!h->is_final && !h->have_labels) return SEG_ERR_STATE;
   seg_status st = SEG_OK;
-  {
-    // fixed staging buffers: rounds x in TF32 mode, pads the pitch, keeps the graph's pointers constant;
-    // the same launch advances the device-side step counter and Adam's bias corrections
-    Launch lc(h, K_COPY);
-    SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
-                                   h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   h->stream), "input staging");
-  }
   if (h->profile || !h->graphs_enabled) {
-    st = enqueue_step(h, batch, !h->profile);
+    st = enqueue_step(h, batch, !h->profile && h->fork_enabled, x, cls, loss_out);
   } else {
     seg_handle::StepGraph& g = h->graphs[batch];
     if (g.exec != nullptr) {
-      SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
-      h->launches += g.kernels;
+      st = replay_graph(h, g, x, cls, loss_out);
     } else if (g.eager_runs == 0) {
-      st = enqueue_step(h, batch, true);      // first step at this batch size: eager (also sets kernel attributes)
+      st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);   // first step at this batch size: eager (sets kernel attributes)
       g.eager_runs = 1;
     } else {
       const uint64_t before = h->launches;
@@ -550,30 +624,34 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
       if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         cudaGetLastError();
         h->graphs_enabled = false;
-        st = enqueue_step(h, batch, true);
+        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);
       } else {
-        st = enqueue_step(h, batch, true);
+        h->capturing = true; h->cap_stage_node = nullptr; h->cap_loss_node = nullptr;
+        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);
+        h->capturing = false;
         cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
-        if (st == SEG_OK && e == cudaSuccess && graph != nullptr &&
-            cudaGraphInstantiate(&g.exec, graph, 0) == cudaSuccess) {
+        if (st == SEG_OK && e == cudaSuccess && graph != nullptr && adopt_captured_graph(h, g, graph)) {
           g.kernels = h->launches - before;
-          SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
+          h->launches = before;
+          st = replay_graph(h, g, x, cls, loss_out);
         } else {
           // capture did not work here: run eagerly from now on
+          if (getenv("SEG_DEBUG"))
+            fprintf(stderr, "seg: step capture failed (status %d, end-capture '%s', nodes %p %p, last '%s')\n", (int)st,
+                    cudaGetErrorString(e), (void*)h->cap_stage_node, (void*)h->cap_loss_node,
+                    cudaGetErrorString(cudaPeekAtLastError()));
           cudaGetLastError();
+          if (graph) cudaGraphDestroy(graph);
           g.exec = nullptr;
           h->graphs_enabled = false;
           h->launches = before;
-          st = enqueue_step(h, batch, true);
+          st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);
         }
-        if (graph) cudaGraphDestroy(graph);
       }
     }
   }
   if (st != SEG_OK) return st;
   ++h->step;
-  if (loss_out)
-    SEG_TRY(h, cudaMemcpyAsync(loss_out, h->loss_slot, sizeof(float), cudaMemcpyDeviceToDevice, h->stream), "loss copy");
   if (y_out && (st = copy_out(h, y_out, batch)) != SEG_OK) return st;
   return SEG_OK;
 }
