@@ -25,11 +25,20 @@
 // CTA j adds what it received and runs the epilogue on that slice).  One SM's shared-memory fill rate bounds a single CTA's main loop, so spreading K over a
 // cluster shortens exactly the part of the kernel that grows with the problem.
 //
+// Large problems use gemm_tc_pair_kernel: two CTAs of a cluster share one 256 x 256 output tile
+// through tcgen05.mma.cta_group::2.  Each CTA stages its own 128 rows of A and its own 128 columns
+// of B (32 KiB per k-block instead of 48 KiB for the same 128 x 256 x 64 of work per SM), which is
+// what matters because the single-CTA kernel is bound by one SM's shared-memory fill rate, not by
+// the tensor pipe.  The even CTA issues the MMAs for the pair; TMA loads of both CTAs complete on
+// the even CTA's "full" barrier; one commit frees the stage in both CTAs.
+//
 // Every wait on an mbarrier is bounded: after about two seconds the waiting thread raises an abort
 // flag, records DEV_TIMEOUT in the status word and all roles leave their loops; TMEM is released
 // before the CTA exits.
 #include <cuda.h>
 #include <stdlib.h>
+
+#include <algorithm>
 
 #include "common.cuh"
 
@@ -641,6 +650,214 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+
+// ---- CTA-pair kernel (tcgen05 cta_group::2) ---------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                                 uint32_t bar_cluster_addr) {
+  // the completion barrier may live in the peer CTA of the pair
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// one arrival on the barrier at the same shared-memory offset in both CTAs of the pair, once all
+// MMAs issued so far have completed
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+template <bool TF32>
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  if constexpr (TF32) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+constexpr int PAIR_TILE_M = 256, PAIR_TILE_N = 256;
+constexpr int PAIR_HALF_N = PAIR_TILE_N / 2;
+constexpr int PAIR_B_BYTES = PAIR_HALF_N * TILE_ROW_BYTES;            // 16 KiB: this CTA's half of B
+constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_BYTES;         // 32 KiB per CTA per k-block
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + SMEM_EXTRA;
+
+template <bool TF32, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    int M, int N, int K, EpilogueArgs epi, int* dev_status) {
+  constexpr int STAGES = PAIR_STAGES;
+  constexpr int BLOCK_K = TF32 ? 32 : 64;
+  constexpr int UMMA_K = TF32 ? 8 : 16;
+  constexpr int CHUNK = TF32 ? 32 : 64;
+  constexpr int MN_CHUNK_BYTES = BLOCK_K * TILE_ROW_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * PAIR_TILE_N;      // two 256-column accumulators per CTA
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * A_TILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * PAIR_STAGE_BYTES);
+  // bars[0..S) full (used in the even CTA), [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty (even CTA)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();             // 0: issues the MMAs of the pair
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }   // 4 warps x 2 CTAs
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();                     // both CTAs' barriers exist before any cross-CTA signal
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m = (M + PAIR_TILE_M - 1) / PAIR_TILE_M;
+  const int tiles_n = (N + PAIR_TILE_N - 1) / PAIR_TILE_N;
+  const int n_tiles = tiles_m * tiles_n;
+  const int num_k = (K + BLOCK_K - 1) / BLOCK_K;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs; completion on the even CTA's barrier) ----------------
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+        const int m0 = (t % tiles_m) * PAIR_TILE_M + (int)rank * BLOCK_M;
+        const int n0 = (t / tiles_m) * PAIR_TILE_N + (int)rank * PAIR_HALF_N;
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(2 * PAIR_STAGE_BYTES));
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
+          const uint32_t a_dst = smem_u32(smem_a + stage * A_TILE_BYTES);
+          const uint32_t b_dst = smem_u32(smem_b + stage * PAIR_B_BYTES);
+          const int k0 = kb * BLOCK_K;
+          if constexpr (A_MN) {
+#pragma unroll
+            for (int c = 0; c < BLOCK_M / CHUNK; ++c)
+              tma_load_2d_pair(a_dst + c * MN_CHUNK_BYTES, &map_a, m0 + c * CHUNK, k0, fb);
+          } else {
+            tma_load_2d_pair(a_dst, &map_a, k0, m0, fb);
+          }
+          if constexpr (B_MN) {
+#pragma unroll
+            for (int c = 0; c < PAIR_HALF_N / CHUNK; ++c)
+              tma_load_2d_pair(b_dst + c * MN_CHUNK_BYTES, &map_b, n0 + c * CHUNK, k0, fb);
+          } else {
+            tma_load_2d_pair(b_dst, &map_b, k0, n0, fb);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: the even CTA only ----------------
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t fmt = TF32 ? 2u : 1u;
+      constexpr uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(PAIR_TILE_N >> 3) << 17) |
+                                 ((uint32_t)(PAIR_TILE_M >> 4) << 24);
+      constexpr uint32_t a_lbo = A_MN ? MN_CHUNK_BYTES : 16, b_lbo = B_MN ? MN_CHUNK_BYTES : 16;
+      constexpr uint32_t a_kstep = A_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      constexpr uint32_t b_kstep = B_MN ? UMMA_K * TILE_ROW_BYTES : 32;
+      constexpr uint32_t a_sbo = (TF32 && A_MN) ? 512 : 1024, b_sbo = (TF32 && B_MN) ? 512 : 1024;
+      constexpr uint32_t a_lay = (TF32 && A_MN) ? 1 : 2, b_lay = (TF32 && B_MN) ? 1 : 2;
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * PAIR_TILE_N);
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, dev_status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = smem_u32(smem_a + stage * A_TILE_BYTES);
+          const uint32_t b_src = smem_u32(smem_b + stage * PAIR_B_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
+            const uint64_t da = make_smem_desc(a_src + kk * a_kstep, a_lbo, a_sbo, a_lay);
+            const uint64_t db = make_smem_desc(b_src + kk * b_kstep, b_lbo, b_sbo, b_lay);
+            tc_mma_pair<TF32>(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit_pair(empty_bar(stage));       // frees this stage in both CTAs
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull_bar(acc));           // accumulator complete, both CTAs' epilogues may drain it
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------- epilogue warps: each CTA drains its own 128 rows ----------------
+    const int quarter = warp & 3;
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+      const int m0 = (t % tiles_m) * PAIR_TILE_M + (int)rank * BLOCK_M;
+      const int n0 = (t / tiles_m) * PAIR_TILE_N;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+#pragma unroll 1
+      for (int c = 0; c < PAIR_TILE_N / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= N) break;
+        float v[32];
+        tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * PAIR_TILE_N + c * 32), v);
+        if (row < M) epilogue_store(epi, v, row, col0, N);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();                   // the pair releases its tensor memory together, after both are done
+  cluster_wait();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -650,6 +867,8 @@ EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
 bool g_init_done = false, g_init_ok = false;
 bool g_allow_splitk = true;
+bool g_allow_pairs = true;
+long g_pair_min_tiles = 96;
 
 // 2-D tensor map over a row-major matrix: `inner` contiguous elements per row, `outer` rows,
 // `row_stride_bytes` between rows; box = box_inner x box_outer; 128-byte swizzle (32-byte atoms
@@ -743,6 +962,47 @@ int pick_split(int M, int N, int K, bool tf32) {
   return best;
 }
 
+template <bool TF32, bool A_MN, bool B_MN>
+cudaError_t launch_pair_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
+                                const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
+  auto kern = gemm_tc_pair_kernel<TF32, A_MN, B_MN>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
+    if (err != cudaSuccess) return err;
+    attr_set = true;
+  }
+  const int tiles = ((g.M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((g.N + PAIR_TILE_N - 1) / PAIR_TILE_N);
+  const int pairs = std::min(tiles, g_num_sms / 2);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = PAIR_SMEM;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, g.M, g.N, g.K, e, dev_status);
+}
+
+template <bool TF32>
+cudaError_t launch_pair_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUtensorMap& mb,
+                               const GemmDesc& g, const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
+  if (!a_mn && !b_mn) return launch_pair_variant<TF32, false, false>(ma, mb, g, e, dev_status, s);
+  if (!a_mn && b_mn) return launch_pair_variant<TF32, false, true>(ma, mb, g, e, dev_status, s);
+  if (a_mn && b_mn) return launch_pair_variant<TF32, true, true>(ma, mb, g, e, dev_status, s);
+  return cudaErrorNotSupported;
+}
+
+// CTA pairs pay off once there are enough 256 x 256 tiles to keep the machine busy.
+bool use_pairs(int M, int N, int K) {
+  if (!g_allow_pairs) return false;
+  if (M < 256 || N < 256 || K < 256) return false;
+  const long tiles = (long)((M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((N + PAIR_TILE_N - 1) / PAIR_TILE_N);
+  return tiles >= g_pair_min_tiles;
+}
+
 int pick_block_n(int M, int N) {
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   int best = 64; long best_cost = -1;
@@ -774,6 +1034,10 @@ bool gemm_tc_init() {
   if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
   const char* env = getenv("SEG_NO_SPLITK");
   if (env && env[0] == '1') g_allow_splitk = false;
+  env = getenv("SEG_NO_PAIRS");
+  if (env && env[0] == '1') g_allow_pairs = false;
+  env = getenv("SEG_PAIR_MIN_TILES");
+  if (env) g_pair_min_tiles = atol(env);
   g_init_ok = g_num_sms > 0;
   return g_init_ok;
 }
@@ -800,7 +1064,8 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   if (a_pitch * (int64_t)esz >= (1ll << 40) || b_pitch * (int64_t)esz >= (1ll << 40)) return cudaErrorNotSupported;
 
   const int split = g_allow_splitk ? pick_split(g.M, g.N, g.K, tf32) : 1;
-  const int block_n = split > 1 ? SPLITK_BLOCK_N : pick_block_n(g.M, g.N);
+  const bool pairs = (split == 1) && use_pairs(g.M, g.N, g.K);
+  const int block_n = split > 1 ? SPLITK_BLOCK_N : (pairs ? PAIR_HALF_N : pick_block_n(g.M, g.N));
   const uint32_t block_k = tf32 ? 32 : 64, chunk = tf32 ? 32 : 64;
   CUtensorMap ma, mb;
   bool ok;
@@ -815,6 +1080,10 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   e.C = g.C; e.ldc = g.ldc; e.c_dt = g.c_dt; e.c_round = g.c_round; e.epi = g.epi; e.relu = g.relu;
   e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
 
+  if (pairs) {
+    return tf32 ? launch_pair_majors<true>(a_mn, b_mn, ma, mb, g, e, dev_status, s)
+                : launch_pair_majors<false>(a_mn, b_mn, ma, mb, g, e, dev_status, s);
+  }
   if (split > 1) {
     return tf32 ? launch_splitk_majors<true>(a_mn, b_mn, ma, mb, g, e, split, dev_status, s)
                 : launch_splitk_majors<false>(a_mn, b_mn, ma, mb, g, e, split, dev_status, s);

@@ -1,0 +1,22 @@
+"""The product kernels are chosen by problem size (persistent single-CTA tiles, cluster split-K for
+small problems, CTA pairs for large ones).  The small parity shapes would never reach the CTA-pair
+kernel or the unsplit kernel on their own, so the tensor-core parity cases are run again in child
+processes with the selection forced through the library's environment switches (read once per
+process, hence the child processes)."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.mark.parametrize("env", [{"SEG_PAIR_MIN_TILES": "1"}, {"SEG_NO_SPLITK": "1", "SEG_NO_PAIRS": "1"},
+                                 {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}])
+def test_tensor_core_cases_with_forced_kernel_selection(env):
+    child_env = dict(os.environ, **env)
+    res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",
+                          "-k", "tensor_core"], cwd=ROOT, env=child_env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-1000:]
