@@ -242,6 +242,35 @@ class Runner:
             seg.close()
 
 
+def unpartitioned_comparison(workload, steps=5):
+    """End-to-end backprop of the unpartitioned network on the same GPU: one final segment spanning
+    every layer (same precision, optimizer, batch).  Returns its device memory and step time."""
+    import torch
+    from paper_2403_11204_b200.binding import Segment
+    w = workload
+    widths = list(w.segments[0].widths)
+    for spec in w.segments[1:]:
+        widths += list(spec.widths[1:])
+    dt = torch.bfloat16 if w.precision == "bf16" else torch.float32
+    seg = Segment(widths, w.n_classes, True, precision=w.precision, optimizer=w.optimizer, lr=w.lr,
+                  momentum=w.momentum, max_batch=w.batch, segment_id=0, init_seed=wl.INIT_SEED)
+    g = torch.Generator(device="cuda").manual_seed(wl.DATA_SEED)
+    x = torch.rand(w.batch, widths[0], generator=g, device="cuda").to(dt)
+    cls = torch.randint(0, w.n_classes, (w.batch,), generator=g, device="cuda", dtype=torch.int32)
+    loss = torch.zeros(1, device="cuda")
+    for _ in range(3):
+        seg.train_step(x, cls, loss)
+    seg.poll()
+    seg.timer_start()
+    for _ in range(steps):
+        seg.train_step(x, cls, loss)
+    seg.timer_stop()
+    ms = seg.timer_ms() / steps
+    mem = seg.mem_bytes()[1]
+    seg.close()
+    return {"layers": len(widths) - 1, "mem_bytes_peak": mem, "ms_per_step": ms}
+
+
 def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples=None):
     """Runs one workload.  full=True adds the end-to-end leg, per-kernel profile and clocks."""
     import torch
@@ -341,6 +370,19 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
     r.close()
     del r
     torch.cuda.empty_cache()
+    if len(w.segments) > 1:
+        try:
+            e2e_net = unpartitioned_comparison(w)
+            seg_peak = max(s_["mem_bytes_peak"] for s_ in out["segments"])
+            out["memory"] = {"largest_segment_bytes": seg_peak, "unpartitioned_bytes": e2e_net["mem_bytes_peak"],
+                             "ratio": e2e_net["mem_bytes_peak"] / seg_peak,
+                             "unpartitioned_ms_per_step": e2e_net["ms_per_step"],
+                             "segments_ms_per_step_sum": sum(s_["ms_per_step"] for s_ in out["segments"]),
+                             "note": "bytes held by the library per handle (parameters, gradients, optimizer state, "
+                                     "operand copy, activations, dZ, staging); segments trained one at a time need only "
+                                     "the largest segment resident"}
+        except Exception as exc:
+            out["memory"] = {"error": repr(exc)[:200]}
     return out
 
 
@@ -420,7 +462,7 @@ def main():
             "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16"}[w.precision], "data": "synthetic",
             "config": config, "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"],
             "roofline": res.get("roofline"), "kernels": res.get("kernels"), "segments": res["segments"],
-            "label_gen_ms": res["label_gen_ms"], "peaks": peaks}
+            "label_gen_ms": res["label_gen_ms"], "memory": res.get("memory"), "peaks": peaks}
     if not args.no_cpu_baseline:
         line["cpu_baseline"], _ = oracle_samples_per_s(w, budget_s=15.0)
     others = {}
@@ -431,7 +473,7 @@ def main():
             r = measure(ow, k, 3, peaks, device_index=local_rank, full=False)
             others[name] = {"samples_per_s": r["samples_per_s"], "ms_per_step": r["ms_per_step"], "steps": k,
                             "precision": ow.precision, "optimizer": ow.optimizer, "batch": ow.batch,
-                            "concurrent_streams": ow.concurrent,
+                            "concurrent_streams": ow.concurrent, "memory": r.get("memory"),
                             "segments": [{kk: s[kk] for kk in ("segment", "ms_per_step", "samples_per_s", "roofline_frac",
                                                                "gemm_tflops", "mem_bytes_peak")} for s in r["segments"]]}
         except Exception as exc:                       # a secondary workload must not cost the headline
