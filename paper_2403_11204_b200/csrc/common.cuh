@@ -17,19 +17,7 @@ enum Round : int { RND_NONE = 0, RND_TF32 = 1, RND_BF16 = 2 };
 enum Epilogue : int {
   EPI_BIAS_ACT = 0,  // forward: + bias[n], optional ReLU
   EPI_MASK = 1,      // dgrad:   * (mask[m][n] > 0)  (mask = stored post-ReLU activation)
-  EPI_PLAIN = 2,     // wgrad:   store the fp32 product
-  EPI_UPDATE = 3     // wgrad:   store the fp32 product and apply the optimizer to the same elements
-};
-
-// Optimizer update fused into the weight-gradient epilogue (tensor-core kernels only).  p, s1, s2 and
-// p_op are laid out exactly like C (same pitch), so element (m, n) of the product updates element
-// (m, n) of every one of them.
-struct FusedUpdate {
-  float* p; float* s1; float* s2;
-  void* p_op; int op_dt; int op_round;
-  int optimizer;
-  float lr, momentum, beta1, beta2, eps;
-  const float* bc;   // device: Adam bias corrections {1-b1^t, 1-b2^t}
+  EPI_PLAIN = 2      // wgrad:   store the fp32 product
 };
 
 // Device status word values (written by kernels that give up a bounded wait).
@@ -50,7 +38,6 @@ struct GemmDesc {
   const float* bias;        // EPI_BIAS_ACT: [N]
   const void* mask;         // EPI_MASK: [M][ldmask] of c_dt
   int64_t ldmask;
-  FusedUpdate upd;          // EPI_UPDATE
 };
 
 // ---- launchers (each returns the cudaError_t of its launch) -------------------------------

@@ -169,7 +169,6 @@ struct EpilogueArgs {
   const float* bias;
   const void* mask;
   int64_t ldmask;
-  FusedUpdate upd;
 };
 
 template <int BLOCK_N>
@@ -180,105 +179,12 @@ struct SmemLayout {
   static constexpr int TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
 };
 
-// Weight-gradient epilogue with the optimizer fused in: g = the fp32 product; dW is stored, and the
-// parameter, its optimizer state and its reduced-precision operand copy at the same position are
-// updated in the same pass (the arithmetic of update_kernel in elementwise.cu).
-__device__ __forceinline__ void epilogue_update(const EpilogueArgs& e, float (&g)[32], int row, int col0,
-                                                int n_total) {
-  const FusedUpdate& u = e.upd;
-  const int n_valid = min(32, n_total - col0);
-  const int64_t off = (int64_t)row * e.ldc + col0;
-  float* dw = reinterpret_cast<float*>(e.C) + off;
-  float* p = u.p + off;
-  float inv_bc1 = 1.f, inv_bc2 = 1.f;
-  if (u.optimizer == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(u.bc); inv_bc2 = 1.0f / __ldg(u.bc + 1); }
-  const bool vec = ((n_valid & 3) == 0) && ((reinterpret_cast<uintptr_t>(dw) & 15u) == 0);
-#pragma unroll
-  for (int j = 0; j < 32; j += 4) {
-    if (j >= n_valid) break;
-    const int cnt = min(4, n_valid - j);
-    float pv[4], mv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
-    if (vec) {
-      const float4 t = *reinterpret_cast<const float4*>(p + j);
-      pv[0] = t.x; pv[1] = t.y; pv[2] = t.z; pv[3] = t.w;
-      if (u.optimizer != SEG_SGD) {
-        const float4 m = *reinterpret_cast<const float4*>(u.s1 + off + j);
-        mv[0] = m.x; mv[1] = m.y; mv[2] = m.z; mv[3] = m.w;
-      }
-      if (u.optimizer == SEG_ADAM) {
-        const float4 v = *reinterpret_cast<const float4*>(u.s2 + off + j);
-        vv[0] = v.x; vv[1] = v.y; vv[2] = v.z; vv[3] = v.w;
-      }
-    } else {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        pv[k] = 0.f;
-        if (k < cnt) {
-          pv[k] = p[j + k];
-          if (u.optimizer != SEG_SGD) mv[k] = u.s1[off + j + k];
-          if (u.optimizer == SEG_ADAM) vv[k] = u.s2[off + j + k];
-        }
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float gk = g[j + k];
-      if (u.optimizer == SEG_SGD) {
-        pv[k] = pv[k] - u.lr * gk;
-      } else if (u.optimizer == SEG_SGD_MOMENTUM) {
-        mv[k] = u.momentum * mv[k] + gk;
-        pv[k] = pv[k] - u.lr * mv[k];
-      } else {
-        mv[k] = u.beta1 * mv[k] + (1.0f - u.beta1) * gk;
-        vv[k] = u.beta2 * vv[k] + (1.0f - u.beta2) * gk * gk;
-        const float mhat = mv[k] * inv_bc1;
-        const float vhat = vv[k] * inv_bc2;
-        pv[k] = pv[k] - u.lr * mhat / (sqrtf(vhat) + u.eps);
-      }
-    }
-    if (vec) {
-      *reinterpret_cast<float4*>(dw + j) = make_float4(g[j], g[j + 1], g[j + 2], g[j + 3]);
-      *reinterpret_cast<float4*>(p + j) = make_float4(pv[0], pv[1], pv[2], pv[3]);
-      if (u.optimizer != SEG_SGD) *reinterpret_cast<float4*>(u.s1 + off + j) = make_float4(mv[0], mv[1], mv[2], mv[3]);
-      if (u.optimizer == SEG_ADAM) *reinterpret_cast<float4*>(u.s2 + off + j) = make_float4(vv[0], vv[1], vv[2], vv[3]);
-      if (u.p_op != nullptr) {
-        if (u.op_dt == DT_BF16) {
-          __nv_bfloat162 lo = __floats2bfloat162_rn(pv[0], pv[1]);
-          __nv_bfloat162 hi = __floats2bfloat162_rn(pv[2], pv[3]);
-          uint2 q;
-          q.x = *reinterpret_cast<uint32_t*>(&lo); q.y = *reinterpret_cast<uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(u.p_op) + off + j) = q;
-        } else {
-          *reinterpret_cast<float4*>(reinterpret_cast<float*>(u.p_op) + off + j) =
-              make_float4(apply_round(pv[0], u.op_round), apply_round(pv[1], u.op_round),
-                          apply_round(pv[2], u.op_round), apply_round(pv[3], u.op_round));
-        }
-      }
-    } else {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (k < cnt) {
-          dw[j + k] = g[j + k];
-          p[j + k] = pv[k];
-          if (u.optimizer != SEG_SGD) u.s1[off + j + k] = mv[k];
-          if (u.optimizer == SEG_ADAM) u.s2[off + j + k] = vv[k];
-          if (u.p_op != nullptr) {
-            if (u.op_dt == DT_BF16) reinterpret_cast<__nv_bfloat16*>(u.p_op)[off + j + k] = __float2bfloat16_rn(pv[k]);
-            else reinterpret_cast<float*>(u.p_op)[off + j + k] = apply_round(pv[k], u.op_round);
-          }
-        }
-      }
-    }
-  }
-}
-
 // Epilogue for up to 32 consecutive columns of one row.  Columns are handled in groups of 8 with
 // 16-byte accesses when the group count is whole and the row segment is 16-byte aligned (every
 // lane touches its own row, so wide accesses are what keeps the number of memory wavefronts down);
 // ragged or unaligned segments fall back to scalar accesses.
 __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], int row, int col0,
                                                int n_total) {
-  if (e.epi == EPI_UPDATE) { epilogue_update(e, v, row, col0, n_total); return; }
   const int n_valid = min(32, n_total - col0);
   const bool whole = (n_valid & 7) == 0;
   if (e.epi == EPI_BIAS_ACT) {
@@ -1172,7 +1078,7 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
 
   EpilogueArgs e;
   e.C = g.C; e.ldc = g.ldc; e.c_dt = g.c_dt; e.c_round = g.c_round; e.epi = g.epi; e.relu = g.relu;
-  e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask; e.upd = g.upd;
+  e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
 
   if (pairs) {
     return tf32 ? launch_pair_majors<true>(a_mn, b_mn, ma, mb, g, e, dev_status, s)

@@ -93,7 +93,6 @@ struct seg_handle {
   bool capturing = false;
   std::map<int, StepGraph> graphs; // by batch size
   bool graphs_enabled = true;
-  bool fuse_update = false;        // optimizer inside the weight-gradient epilogue (opt-in: SEG_FUSE_UPDATE=1)
   bool fork_enabled = true;        // run the gradient and update branches on their own streams
   float* sil = nullptr;
   bool have_labels = false;
@@ -179,7 +178,6 @@ seg_status run_gemm(seg_handle* h, const GemmDesc& g_in, int kind, cudaStream_t 
     if (e != cudaErrorNotSupported) return fail_cuda(h, e, "tensor-core product launch");
     cudaGetLastError();
   }
-  if (g.epi == EPI_UPDATE) g.epi = EPI_PLAIN;     // the FFMA kernels leave the update to update_kernel
   SEG_TRY(h, launch_gemm_simt(g, stream), "FFMA product launch");
   return SEG_OK;
 }
@@ -389,8 +387,6 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   {
     const char* env = getenv("SEG_NO_GRAPH");
     if (env && env[0] == '1') h->graphs_enabled = false;
-    env = getenv("SEG_FUSE_UPDATE");
-    if (env && env[0] == '1') h->fuse_update = true;
     env = getenv("SEG_NO_FORK");
     if (env && env[0] == '1') h->fork_enabled = false;
   }
@@ -526,9 +522,7 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
       if ((st = run_gemm(h, d, K_DGRAD, mainst)) != SEG_OK) return st;
       if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[l - 1], mainst), "event record");
     }
-    // gradient branch: bias gradient and weight gradient of layer l (need dZ_l).  With the optimizer
-    // fused into the weight-gradient epilogue the product also rewrites W_l, so it waits for dgrad(l).
-    const bool fuse = h->fuse_update && h->use_tc;
+    // gradient branch: bias gradient and weight gradient of layer l (need dZ_l)
     if (forked) SEG_TRY(h, cudaStreamWaitEvent(side, h->ev_dz[l], 0), "stream wait");
     {
       Launch lb(h, K_BIAS, side);
@@ -541,27 +535,15 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
     w.A = dz_l; w.a_sm = 1; w.a_sk = ld_dz; w.a_dt = h->act_dt;
     w.B = a_prev; w.b_sk = ld_prev; w.b_sn = 1; w.b_dt = h->act_dt;
     w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
-    w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = fuse ? EPI_UPDATE : EPI_PLAIN;
-    if (fuse) {
-      w.upd.p = h->params + lo;
-      w.upd.s1 = h->state1 ? h->state1 + lo : nullptr; w.upd.s2 = h->state2 ? h->state2 + lo : nullptr;
-      w.upd.p_op = h->params_op ? (void*)(reinterpret_cast<char*>(h->params_op) + lo * elem_size(h->op_dt)) : nullptr;
-      w.upd.op_dt = h->op_dt; w.upd.op_round = h->op_round; w.upd.optimizer = h->optimizer;
-      w.upd.lr = h->lr; w.upd.momentum = h->momentum; w.upd.beta1 = h->beta1; w.upd.beta2 = h->beta2;
-      w.upd.eps = h->eps; w.upd.bc = h->bc_dev;
-      if (forked && l > 0) SEG_TRY(h, cudaStreamWaitEvent(side, h->ev_dz[l - 1], 0), "stream wait");   // dgrad(l) done
-    }
-    bool fused_done = false;
-    if ((st = run_gemm(h, w, K_WGRAD, side, &fused_done)) != SEG_OK) return st;
-    fused_done = fused_done && fuse;
+    w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
+    if ((st = run_gemm(h, w, K_WGRAD, side)) != SEG_OK) return st;
     if (forked) SEG_TRY(h, cudaEventRecord(h->ev_wg[l], side), "event record");
-    // update branch: what the product did not update itself (the bias; or the whole layer, W_l and b_l
-    // being adjacent in the flat range)
+    // update branch: layer l's tensors (W_l and b_l are adjacent in the flat range)
     if (forked) {
       SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_wg[l], 0), "stream wait");
       if (l > 0) SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_dz[l - 1], 0), "stream wait");   // dgrad(l) done
     }
-    const int64_t ulo = fused_done ? Ly.b_off : lo;
+    const int64_t ulo = lo;
     UpdateArgs u{};
     u.p = h->params + ulo; u.g = h->grads + ulo;
     u.s1 = h->state1 ? h->state1 + ulo : nullptr; u.s2 = h->state2 ? h->state2 + ulo : nullptr;
