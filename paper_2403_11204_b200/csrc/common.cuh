@@ -90,6 +90,28 @@ cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* s
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2, cudaStream_t s);
 
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Kernels of one stream are launched with programmatic stream serialisation: a kernel may become
+// resident and run its prologue while its predecessor drains.  Every kernel therefore calls
+// pdl_wait() before its first access to global memory (it returns once the predecessor grid has
+// completed and its writes are visible; a no-op for ordinary launches) and pdl_trigger() to let its
+// own successor start early.
+extern bool g_use_pdl;
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                            Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // ---- small device helpers ------------------------------------------------------------------
 __device__ __forceinline__ float round_tf32_rne(float x) {
   uint32_t u = __float_as_uint(x);

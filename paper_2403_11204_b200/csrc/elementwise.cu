@@ -5,6 +5,9 @@
 #include "common.cuh"
 
 namespace segk {
+
+bool g_use_pdl = true;
+
 namespace {
 
 constexpr int kLossThreads = 256;
@@ -69,6 +72,8 @@ mse_loss_kernel(const TOut* __restrict__ out, int64_t ld_out, const int32_t* __r
                 const float* __restrict__ sil, int n_p, int batch, int relu_mask,
                 TDz* __restrict__ dz, int dz_round, int64_t ld_dz, float* partials,
                 unsigned int* counter, float* loss_out) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[32];
   const int64_t total = (int64_t)batch * n_p;
   const float gscale = 2.0f / (float)total;
@@ -99,6 +104,8 @@ __global__ void __launch_bounds__(kLossThreads)
 softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* __restrict__ cls,
                   int n_classes, int batch, int relu_mask, TDz* __restrict__ dz, int dz_round,
                   int64_t ld_dz, float* partials, unsigned int* counter, float* loss_out) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[32];
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
@@ -138,6 +145,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 bias_grad_kernel(const T* __restrict__ dz, int64_t ld, int batch, int n, float* __restrict__ db,
                  float* __restrict__ scratch, unsigned int* __restrict__ counters) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float part[8][33];
   __shared__ bool is_last;
   const int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
@@ -186,6 +195,8 @@ bias_grad_kernel(const T* __restrict__ dz, int64_t ld, int batch, int n, float* 
 template <int OPT, int OPDT>
 __global__ void __launch_bounds__(256)
 update_kernel(UpdateArgs u) {
+  pdl_wait();
+  pdl_trigger();
   const int64_t n4 = u.n >> 2;
   float4* __restrict__ p4 = reinterpret_cast<float4*>(u.p);
   const float4* __restrict__ g4 = reinterpret_cast<const float4*>(u.g);
@@ -246,6 +257,8 @@ update_kernel(UpdateArgs u) {
 __global__ void __launch_bounds__(256)
 copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt, int64_t ld_src,
               int rows, int cols, int round) {
+  pdl_wait();
+  pdl_trigger();
   const int64_t total = (int64_t)rows * cols;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
        e += (int64_t)gridDim.x * blockDim.x) {
@@ -259,6 +272,8 @@ __global__ void __launch_bounds__(256)
 stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows, int cols,
                     int round, int32_t* cls_dst, const int32_t* cls_src, unsigned long long* t, float* bc,
                     float beta1, float beta2) {
+  pdl_wait();
+  pdl_trigger();
   const int64_t total = (int64_t)rows * cols;
   const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (tid == 0 && t != nullptr) {           // step counter and Adam bias corrections of this step
@@ -291,11 +306,11 @@ cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const i
                             unsigned int* counter, float* loss_out, cudaStream_t s) {
   const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
   if (out_dt == DT_BF16 && dz_dt == DT_BF16) {
-    mse_loss_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, kLossThreads, 0, s>>>(
+    launch_k(mse_loss_kernel<__nv_bfloat16, __nv_bfloat16>, dim3(grid), dim3(kLossThreads), 0, s, 
         (const __nv_bfloat16*)out, ld_out, cls, sil, n_p, batch, relu_mask, (__nv_bfloat16*)dz,
         dz_round, ld_dz, partials, counter, loss_out);
   } else if (out_dt == DT_F32 && dz_dt == DT_F32) {
-    mse_loss_kernel<float, float><<<grid, kLossThreads, 0, s>>>(
+    launch_k(mse_loss_kernel<float, float>, dim3(grid), dim3(kLossThreads), 0, s, 
         (const float*)out, ld_out, cls, sil, n_p, batch, relu_mask, (float*)dz, dz_round, ld_dz,
         partials, counter, loss_out);
   } else {
@@ -311,11 +326,11 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
   const int warps = kLossThreads / 32;
   const int grid = grid_for(batch, warps, kMaxLossBlocks);
   if (dz_dt == DT_BF16) {
-    softmax_ce_kernel<__nv_bfloat16><<<grid, kLossThreads, 0, s>>>(
+    launch_k(softmax_ce_kernel<__nv_bfloat16>, dim3(grid), dim3(kLossThreads), 0, s, 
         logits, ld_logits, cls, n_classes, batch, relu_mask, (__nv_bfloat16*)dz, dz_round, ld_dz,
         partials, counter, loss_out);
   } else {
-    softmax_ce_kernel<float><<<grid, kLossThreads, 0, s>>>(logits, ld_logits, cls, n_classes,
+    launch_k(softmax_ce_kernel<float>, dim3(grid), dim3(kLossThreads), 0, s, logits, ld_logits, cls, n_classes,
                                                           batch, relu_mask, (float*)dz, dz_round,
                                                           ld_dz, partials, counter, loss_out);
   }
@@ -335,9 +350,9 @@ cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, i
   const int chunks = (batch + kBiasRowsPerChunk - 1) / kBiasRowsPerChunk;
   dim3 grid((n + 31) / 32, (partials == nullptr || counters == nullptr) ? 1 : chunks);
   if (dz_dt == DT_BF16)
-    bias_grad_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)dz, ld, batch, n, db, partials, counters);
+    launch_k(bias_grad_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, s, (const __nv_bfloat16*)dz, ld, batch, n, db, partials, counters);
   else
-    bias_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dz, ld, batch, n, db, partials, counters);
+    launch_k(bias_grad_kernel<float>, dim3(grid), dim3(256), 0, s, (const float*)dz, ld, batch, n, db, partials, counters);
   return cudaGetLastError();
 }
 
@@ -347,8 +362,8 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
   const int grid = grid_for(u.n >> 2, 256, 148 * 8);
   const bool bf = (u.p_op != nullptr && u.op_dt == DT_BF16);
 #define SEGK_UPD(OPT)                                                      \
-  if (bf) update_kernel<OPT, DT_BF16><<<grid, 256, 0, s>>>(u);             \
-  else update_kernel<OPT, DT_F32><<<grid, 256, 0, s>>>(u)
+  if (bf) launch_k(update_kernel<OPT, DT_BF16>, dim3(grid), dim3(256), 0, s, u);             \
+  else launch_k(update_kernel<OPT, DT_F32>, dim3(grid), dim3(256), 0, s, u)
   switch (u.optimizer) {
     case SEG_SGD: SEGK_UPD(SEG_SGD); break;
     case SEG_SGD_MOMENTUM: SEGK_UPD(SEG_SGD_MOMENTUM); break;
@@ -363,7 +378,7 @@ cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* s
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2, cudaStream_t s) {
   const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
-  stage_inputs_kernel<<<grid, 256, 0, s>>>(dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
+  launch_k(stage_inputs_kernel, dim3(grid), dim3(256), 0, s, dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
                                            beta1, beta2);
   return cudaGetLastError();
 }
@@ -372,7 +387,7 @@ cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src
                           int64_t ld_src, int rows, int cols, int round, cudaStream_t s) {
   if ((int64_t)rows * cols == 0) return cudaSuccess;
   const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
-  copy2d_kernel<<<grid, 256, 0, s>>>(dst, dst_dt, ld_dst, src, src_dt, ld_src, rows, cols, round);
+  launch_k(copy2d_kernel, dim3(grid), dim3(256), 0, s, dst, dst_dt, ld_dst, src, src_dt, ld_src, rows, cols, round);
   return cudaGetLastError();
 }
 

@@ -18,6 +18,8 @@ __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return _
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(GemmDesc g) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ __align__(16) float As[BK][BM + PAD];
   __shared__ __align__(16) float Bs[BK][BN + PAD];
   const TIn* __restrict__ A = reinterpret_cast<const TIn*>(g.A);
@@ -88,11 +90,11 @@ cudaError_t launch_gemm_simt(const GemmDesc& g, cudaStream_t s) {
   if (g.M <= 0 || g.N <= 0) return cudaSuccess;
   if (g.a_dt != g.b_dt) return cudaErrorInvalidValue;
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
-  if (g.a_dt == DT_F32 && g.c_dt == DT_F32) gemm_simt_kernel<float, float><<<grid, 256, 0, s>>>(g);
+  if (g.a_dt == DT_F32 && g.c_dt == DT_F32) launch_k(gemm_simt_kernel<float, float>, dim3(grid), dim3(256), 0, s, g);
   else if (g.a_dt == DT_BF16 && g.c_dt == DT_BF16)
-    gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, s>>>(g);
+    launch_k(gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16>, dim3(grid), dim3(256), 0, s, g);
   else if (g.a_dt == DT_BF16 && g.c_dt == DT_F32)
-    gemm_simt_kernel<__nv_bfloat16, float><<<grid, 256, 0, s>>>(g);
+    launch_k(gemm_simt_kernel<__nv_bfloat16, float>, dim3(grid), dim3(256), 0, s, g);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }

@@ -326,6 +326,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                         // everything above overlapped the previous kernel's tail
+  pdl_trigger();
 
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   const int tiles_n = (N + BLOCK_N - 1) / BLOCK_N;
@@ -512,6 +514,8 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   cluster_arrive();                   // "my barriers are initialised"; the matching wait sits in front of the
   tc_fence_after();                   // first remote access (the slice exchange), off the main loop's path
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_trigger();
 
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   const int tile = blockIdx.x / split;
@@ -741,6 +745,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   cluster_wait();                     // both CTAs' barriers exist before any cross-CTA signal
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_trigger();
 
   const int tiles_m = (M + PAIR_TILE_M - 1) / PAIR_TILE_M;
   const int tiles_n = (N + PAIR_TILE_N - 1) / PAIR_TILE_N;
@@ -900,8 +906,7 @@ cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const G
   }
   const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + BLOCK_N - 1) / BLOCK_N);
   const int grid = tiles < g_num_sms ? tiles : g_num_sms;
-  kern<<<grid, NUM_THREADS, L::TOTAL, s>>>(ma, mb, g.M, g.N, g.K, e, dev_status);
-  return cudaGetLastError();
+  return launch_k(kern, dim3(grid), dim3(NUM_THREADS), L::TOTAL, s, ma, mb, g.M, g.N, g.K, e, dev_status);
 }
 
 template <bool TF32, int BLOCK_N>
@@ -930,10 +935,12 @@ cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, 
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = SPLITK_SMEM;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, kern, ma, mb, g.M, g.N, g.K, split, e, dev_status);
 }
 
@@ -979,10 +986,12 @@ cudaError_t launch_pair_variant(const CUtensorMap& ma, const CUtensorMap& mb, co
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = PAIR_SMEM;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, kern, ma, mb, g.M, g.N, g.K, e, dev_status);
 }
 

@@ -107,6 +107,8 @@ enum Transform : int { TR_UNIFORM_SCALED = 0, TR_NORMAL = 1, TR_SYMMETRIC = 2 };
 __global__ void __launch_bounds__(256)
 fill_random_kernel(float* __restrict__ dst, int64_t n_elems, int cols, int64_t ld, uint32_t k0,
                    uint32_t k1, uint32_t segment_id, uint32_t stream, int transform, float scale) {
+  pdl_wait();
+  pdl_trigger();
   const int64_t n_blocks = (n_elems + 3) / 4;
   for (int64_t q = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; q < n_blocks;
        q += (int64_t)gridDim.x * blockDim.x) {
@@ -139,7 +141,7 @@ cudaError_t fill(float* dst, int rows, int cols, int64_t ld, uint64_t seed, int 
   if (n == 0) return cudaSuccess;
   const int64_t blocks = ((n + 3) / 4 + 255) / 256;
   const int grid = (int)(blocks < 148 * 8 ? blocks : 148 * 8);
-  fill_random_kernel<<<grid, 256, 0, s>>>(dst, n, cols, ld, (uint32_t)(seed & 0xFFFFFFFFull),
+  launch_k(fill_random_kernel, dim3(grid), dim3(256), 0, s, dst, n, cols, ld, (uint32_t)(seed & 0xFFFFFFFFull),
                                           (uint32_t)(seed >> 32), (uint32_t)segment_id, stream,
                                           transform, scale);
   return cudaGetLastError();

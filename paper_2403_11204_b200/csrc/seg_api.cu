@@ -387,6 +387,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   {
     const char* env = getenv("SEG_NO_GRAPH");
     if (env && env[0] == '1') h->graphs_enabled = false;
+    env = getenv("SEG_NO_PDL");
+    if (env && env[0] == '1') g_use_pdl = false;
     env = getenv("SEG_NO_FORK");
     if (env && env[0] == '1') h->fork_enabled = false;
   }

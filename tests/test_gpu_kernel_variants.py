@@ -14,7 +14,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 @pytest.mark.parametrize("env", [{"SEG_PAIR_MIN_TILES": "1"}, {"SEG_NO_SPLITK": "1", "SEG_NO_PAIRS": "1"},
-                                 {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}])
+                                 {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}, {"SEG_NO_PDL": "1"}])
 def test_tensor_core_cases_with_forced_kernel_selection(env):
     child_env = dict(os.environ, **env)
     res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",
