@@ -524,13 +524,8 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
       if ((st = run_gemm(h, d, K_DGRAD, mainst)) != SEG_OK) return st;
       if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[l - 1], mainst), "event record");
     }
-    // gradient branch: bias gradient and weight gradient of layer l (need dZ_l)
+    // gradient branch: weight gradient of layer l (needs dZ_l)
     if (forked) SEG_TRY(h, cudaStreamWaitEvent(side, h->ev_dz[l], 0), "stream wait");
-    {
-      Launch lb(h, K_BIAS, side);
-      SEG_TRY(h, launch_bias_grad(dz_l, h->act_dt, ld_dz, batch, Ly.out, h->grads + Ly.b_off, h->bias_scratch,
-                                  h->bias_counters, side), "bias gradient");
-    }
     const int64_t lo = Ly.w_off;
     const int64_t hi = (l + 1 < L) ? h->layers[l + 1].w_off : h->n_flat;
     GemmDesc w{};
@@ -540,7 +535,14 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
     w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
     if ((st = run_gemm(h, w, K_WGRAD, side)) != SEG_OK) return st;
     if (forked) SEG_TRY(h, cudaEventRecord(h->ev_wg[l], side), "event record");
-    // update branch: layer l's tensors (W_l and b_l are adjacent in the flat range)
+    // update branch: the bias gradient (needs dZ_l only, so it runs beside the weight-gradient product),
+    // then the update of layer l's tensors (W_l and b_l are adjacent in the flat range)
+    if (forked) SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_dz[l], 0), "stream wait");
+    {
+      Launch lb(h, K_BIAS, upd);
+      SEG_TRY(h, launch_bias_grad(dz_l, h->act_dt, ld_dz, batch, Ly.out, h->grads + Ly.b_off, h->bias_scratch,
+                                  h->bias_counters, upd), "bias gradient");
+    }
     if (forked) {
       SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_wg[l], 0), "stream wait");
       if (l > 0) SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_dz[l - 1], 0), "stream wait");   // dgrad(l) done
