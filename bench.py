@@ -437,10 +437,11 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2403_11204_b200 import build
-    if rank == 0 or world == 1:
-        build.build()
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()                                   # in-tree library; a no-op when it is up to date
+    if world > 1:
         dist.barrier()
     peaks = load_peaks()
     res = measure(w, args.steps, args.warmup, peaks, device_index=local_rank, full=True,
