@@ -31,6 +31,11 @@ from paper_2403_11204_b200 import workloads as wl
 
 L2_BYTES = 126 * 1024 * 1024
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel kind, from the
+# ncu capture summarised in profiles/gemm_tc_splitk_paper_shaped.md (forward products of segment 1; average
+# of the three captured launches).  Workloads without a capture of their dominant kind report null.
+NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): 2.26e6}
+
 
 # ---- peaks -----------------------------------------------------------------------------------
 def load_peaks():
@@ -338,7 +343,7 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
         if v["flops"] > 0:
             achieved = v["flops"] / (v["ms"] * 1e-3) / 1e12
             out["roofline"] = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": tp, "unit": "TFLOP/s",
-                               "frac": achieved / tp, "traffic": None,
+                               "frac": achieved / tp, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
                                "peak_source": f"{peaks['source']}: sustained bf16 {peaks['bf16_tflops_sustained']} TF/s"
                                               + (" x 0.5 nominal TF32 ratio" if w.precision == "tf32" else ""),
                                "timing": "CUDA events around every launch of this kind, same steps re-run after the timed region",
