@@ -372,6 +372,22 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
         h2d = sum(w.batch * (spec.widths[0] * (2 if w.precision == "bf16" else 4) + 4) for spec in w.segments)
         out["e2e"] = {"value": e_steps * w.batch / dt, "unit": "samples/s", "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": 4 * len(w.segments), "steps": e_steps}
+    if full and not w.concurrent:
+        # the whole procedure of Section 2, one epoch per segment: train segment k over the resident set in
+        # stored order (last partial batch included), store its response, hand it to segment k+1
+        from paper_2403_11204_b200 import binding
+        n_all = r.x[0].shape[0] + 0
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        binding.train_partitioned(r.segs, r.x[0], r.cls, w.batch, [1] * len(r.segs))
+        e1.record()
+        torch.cuda.synchronize()
+        ms_proc = e0.elapsed_time(e1)
+        out["procedure"] = {"what": "one epoch per segment over the resident set, in order, response of each segment "
+                                    "stored for the next (seg_train_epochs + seg_forward_dataset)",
+                            "samples": n_all, "ms": ms_proc,
+                            "samples_per_s": n_all / (ms_proc * 1e-3)}
     r.close()
     del r
     torch.cuda.empty_cache()
@@ -468,7 +484,8 @@ def main():
             "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16"}[w.precision], "data": "synthetic",
             "config": config, "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"],
             "roofline": res.get("roofline"), "kernels": res.get("kernels"), "segments": res["segments"],
-            "label_gen_ms": res["label_gen_ms"], "memory": res.get("memory"), "peaks": peaks}
+            "label_gen_ms": res["label_gen_ms"], "memory": res.get("memory"), "procedure": res.get("procedure"),
+            "peaks": peaks}
     if not args.no_cpu_baseline:
         line["cpu_baseline"], _ = oracle_samples_per_s(w, budget_s=15.0)
     others = {}

@@ -140,6 +140,20 @@ SEG_API seg_status seg_train_step_host(seg_handle* h, const void* x_host, const 
  *   segment, bf16 for a non-final BF16 segment.                                           */
 SEG_API seg_status seg_forward(seg_handle* h, const void* x, int32_t batch, void* y);
 
+/* Epoch driver (Section 2, both phases): trains the segment for `epochs` passes over a
+ * device-resident data set, in the stored order - the method does not shuffle -, in steps
+ * of `batch` samples; a last partial batch is a smaller step (its means run over its own
+ * size).  x [n][widths[0]] and cls [n] as for seg_train_step; losses, if not NULL, is a
+ * device array that receives the loss of every step, epochs * ceil(n / batch) floats.
+ * Equivalent to calling seg_train_step in that order; nothing synchronises.               */
+SEG_API seg_status seg_train_epochs(seg_handle* h, const void* x, const int32_t* cls, int64_t n,
+                                    int32_t batch, int32_t epochs, float* losses);
+
+/* The stored response of a trained segment over a whole data set (Section 2: the left
+ * partition's final response, which is the next partition's input): seg_forward over
+ * consecutive chunks of `batch` rows.  y [n][widths[n_layers]], dtype as for seg_forward. */
+SEG_API seg_status seg_forward_dataset(seg_handle* h, const void* x, int64_t n, int32_t batch, void* y);
+
 /* Frees everything the handle owns.  Synchronises the handle's stream first.             */
 SEG_API seg_status seg_destroy(seg_handle* h);
 

@@ -38,6 +38,8 @@ EXPORTS = {
     "seg_train_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
     "seg_train_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_float)]),
     "seg_forward": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p]),
+    "seg_train_epochs": (c_int32, [c_void_p, c_void_p, c_void_p, ctypes.c_int64, c_int32, c_int32, c_void_p]),
+    "seg_forward_dataset": (c_int32, [c_void_p, c_void_p, ctypes.c_int64, c_int32, c_void_p]),
     "seg_destroy": (c_int32, [c_void_p]),
     "seg_get_labels": (c_int32, [c_void_p, c_void_p]),
     "seg_set_labels": (c_int32, [c_void_p, c_void_p]),
@@ -109,6 +111,35 @@ def label_loss_noalloc(out, cls, sil, relu_mask, dz, loss_out, stream=None):
                                         int(bool(relu_mask)), _ptr(dz), _ptr(loss_out), c_void_p(st.cuda_stream))
     if status != SEG_OK:
         raise SegError(status, "seg_label_loss_noalloc")
+
+
+def train_partitioned(segments, x, cls, batch, epochs):
+    """The paper's training procedure (Section 2, two or more partitions): segment k is trained for
+    epochs[k] passes on the stored response of segment k-1 (segment 0 on x) against its own
+    intermediate labels - the last segment against the class labels - and only then is its response
+    over the whole set computed and handed to segment k+1.  Returns the per-step losses of every
+    segment (device tensors) and the last segment's input.  Marshalling only: every step runs in
+    seg_train_epochs / seg_forward_dataset."""
+    import torch
+    losses = []
+    cur = x
+    for k, (seg, n_ep) in enumerate(zip(segments, epochs)):
+        steps = n_ep * (-(-cur.shape[0] // batch))
+        l = torch.zeros(max(steps, 1), device="cuda")
+        seg.train_epochs(cur, cls, batch, n_ep, l)
+        losses.append(l[:steps])
+        if k + 1 < len(segments):
+            cur = seg.forward_dataset(cur, batch)
+    return losses, cur
+
+
+def predict(segments, x, batch):
+    """The joined network (Section 2: the partitions are joined after training): class = argmax of the
+    last segment's logits."""
+    cur = x
+    for seg in segments:
+        cur = seg.forward_dataset(cur, batch)
+    return cur.argmax(dim=1)
 
 
 class Segment:
@@ -194,6 +225,24 @@ class Segment:
             y = self._empty(batch, self.widths[-1], dtype=self.out_dtype)
         self._check(self.lib.seg_forward(self.h, _ptr(x), batch, _ptr(y)), "seg_forward")
         self.last_batch = batch
+        return y
+
+    def train_epochs(self, x, cls, batch, epochs, losses=None):
+        """seg_train_epochs: `epochs` passes over the resident data set in stored order (no shuffling)."""
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.act_dtype and x.shape[1] == self.widths[0]
+        assert cls.is_cuda and cls.is_contiguous() and cls.dtype == self._torch.int32 and cls.shape[0] == x.shape[0]
+        self._check(self.lib.seg_train_epochs(self.h, _ptr(x), _ptr(cls), x.shape[0], int(batch), int(epochs),
+                                              _ptr(losses)), "seg_train_epochs")
+        self.last_batch = x.shape[0] % batch or batch
+
+    def forward_dataset(self, x, batch, y=None):
+        """seg_forward_dataset: the segment's stored response over the whole set."""
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.act_dtype and x.shape[1] == self.widths[0]
+        if y is None:
+            y = self._empty(x.shape[0], self.widths[-1], dtype=self.out_dtype)
+        self._check(self.lib.seg_forward_dataset(self.h, _ptr(x), x.shape[0], int(batch), _ptr(y)),
+                    "seg_forward_dataset")
+        self.last_batch = x.shape[0] % batch or batch
         return y
 
     # -- inspection -------------------------------------------------------------------------

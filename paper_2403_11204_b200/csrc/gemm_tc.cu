@@ -870,7 +870,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
-int g_num_sms = 0;
+int g_num_sms = 0;      // every device of one process is assumed to be the same part
+
+int current_device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  return dev;
+}
 bool g_init_done = false, g_init_ok = false;
 bool g_allow_splitk = true;
 bool g_allow_pairs = true;
@@ -898,7 +904,8 @@ cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const G
                            const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   using L = SmemLayout<BLOCK_N>;
   auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N>;
-  static bool attr_set = false;
+  static bool attr_set_dev[64] = {};      // the attribute is per device
+  bool& attr_set = attr_set_dev[current_device_slot()];
   if (!attr_set) {
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
     if (err != cudaSuccess) return err;
@@ -923,7 +930,8 @@ template <bool TF32, bool A_MN, bool B_MN>
 cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                                   const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
   auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN>;
-  static bool attr_set = false;
+  static bool attr_set_dev[64] = {};      // the attribute is per device
+  bool& attr_set = attr_set_dev[current_device_slot()];
   if (!attr_set) {
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SPLITK_SMEM);
     if (err != cudaSuccess) return err;
@@ -973,7 +981,8 @@ template <bool TF32, bool A_MN, bool B_MN>
 cudaError_t launch_pair_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                                 const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   auto kern = gemm_tc_pair_kernel<TF32, A_MN, B_MN>;
-  static bool attr_set = false;
+  static bool attr_set_dev[64] = {};      // the attribute is per device
+  bool& attr_set = attr_set_dev[current_device_slot()];
   if (!attr_set) {
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
     if (err != cudaSuccess) return err;

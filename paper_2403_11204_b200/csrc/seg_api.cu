@@ -662,6 +662,39 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
   return SEG_OK;
 }
 
+seg_status seg_train_epochs(seg_handle* h, const void* x, const int32_t* cls, int64_t n, int32_t batch,
+                            int32_t epochs, float* losses) {
+  if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
+  if (n < 1 || epochs < 0) return SEG_ERR_SHAPE;
+  if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
+  const size_t row_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
+  int64_t step = 0;
+  for (int e = 0; e < epochs; ++e) {
+    for (int64_t i = 0; i < n; i += batch, ++step) {
+      const int b = (int)std::min<int64_t>(batch, n - i);
+      seg_status st = seg_train_step(h, reinterpret_cast<const char*>(x) + (size_t)i * row_bytes, cls + i, b,
+                                     losses ? losses + step : nullptr, nullptr);
+      if (st != SEG_OK) return st;
+    }
+  }
+  return SEG_OK;
+}
+
+seg_status seg_forward_dataset(seg_handle* h, const void* x, int64_t n, int32_t batch, void* y) {
+  if (!h || !x || !y) return SEG_ERR_INVALID_ARG;
+  if (n < 1) return SEG_ERR_SHAPE;
+  if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
+  const size_t in_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
+  const size_t out_bytes = (size_t)h->widths[h->n_layers] * elem_size(h->act_dtype[h->n_layers]);
+  for (int64_t i = 0; i < n; i += batch) {
+    const int b = (int)std::min<int64_t>(batch, n - i);
+    seg_status st = seg_forward(h, reinterpret_cast<const char*>(x) + (size_t)i * in_bytes, b,
+                                reinterpret_cast<char*>(y) + (size_t)i * out_bytes);
+    if (st != SEG_OK) return st;
+  }
+  return SEG_OK;
+}
+
 seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t* cls_host, int32_t batch,
                                float* loss_host) {
   if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
