@@ -154,6 +154,18 @@ SEG_API seg_status seg_train_epochs(seg_handle* h, const void* x, const int32_t*
  * consecutive chunks of `batch` rows.  y [n][widths[n_layers]], dtype as for seg_forward. */
 SEG_API seg_status seg_forward_dataset(seg_handle* h, const void* x, int64_t n, int32_t batch, void* y);
 
+/* Recovery step (Section 5, "recovery epochs"): after both partitions are trained, the
+ * left one is trained some more THROUGH the right one, whose weights stay frozen.  Runs
+ * left forward, right forward on the left output, softmax cross-entropy on the class
+ * labels, backprop through the right segment down to its input (no weight gradient, no
+ * update there), then the usual backward pass and optimizer update of the left segment.
+ * left must be non-final and right final, widths must chain, precision and stream must be
+ * the same (SEG_ERR_STATE / SEG_ERR_SHAPE / SEG_ERR_UNSUPPORTED otherwise).  x, cls, batch,
+ * loss_out as for seg_train_step; the loss is the joined network's.  The left segment's
+ * intermediate labels are not used.                                                        */
+SEG_API seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x,
+                                     const int32_t* cls, int32_t batch, float* loss_out);
+
 /* Frees everything the handle owns.  Synchronises the handle's stream first.             */
 SEG_API seg_status seg_destroy(seg_handle* h);
 

@@ -38,6 +38,7 @@ EXPORTS = {
     "seg_train_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
     "seg_train_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_float)]),
     "seg_forward": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p]),
+    "seg_recovery_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_train_epochs": (c_int32, [c_void_p, c_void_p, c_void_p, ctypes.c_int64, c_int32, c_int32, c_void_p]),
     "seg_forward_dataset": (c_int32, [c_void_p, c_void_p, ctypes.c_int64, c_int32, c_void_p]),
     "seg_destroy": (c_int32, [c_void_p]),
@@ -131,6 +132,15 @@ def train_partitioned(segments, x, cls, batch, epochs):
         if k + 1 < len(segments):
             cur = seg.forward_dataset(cur, batch)
     return losses, cur
+
+
+def recovery_step(left, right, x, cls, loss_out=None):
+    """seg_recovery_step: one step of the paper's recovery phase (left trained through the frozen right)."""
+    assert x.is_cuda and x.is_contiguous() and x.dtype == left.act_dtype and x.shape[1] == left.widths[0]
+    assert cls.is_cuda and cls.is_contiguous() and cls.shape[0] == x.shape[0]
+    left._check(left.lib.seg_recovery_step(left.h, right.h, _ptr(x), _ptr(cls), x.shape[0], _ptr(loss_out)),
+                "seg_recovery_step")
+    left.last_batch = right.last_batch = x.shape[0]
 
 
 def predict(segments, x, batch):

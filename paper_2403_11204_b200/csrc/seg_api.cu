@@ -474,12 +474,12 @@ static cudaGraphNode_t last_captured_node(seg_handle* h) {
   return deps[0];
 }
 
+static seg_status enqueue_backward(seg_handle* h, int batch, bool forked);
+
 static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void* x, const int32_t* cls,
                                float* loss_out) {
   const int L = h->n_layers;
   cudaStream_t mainst = h->stream;
-  cudaStream_t side = forked ? h->side : mainst;
-  cudaStream_t upd = forked ? h->upd : mainst;
   seg_status st;
   float* loss_dst = loss_out ? loss_out : h->loss_slot;
   {
@@ -506,6 +506,16 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
     }
   }
   if (h->capturing) h->cap_loss_node = last_captured_node(h);
+  return enqueue_backward(h, batch, forked);
+}
+
+// Backward pass and update of every layer, starting from dZ of the last layer in dzbuf[L-1].
+static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
+  const int L = h->n_layers;
+  cudaStream_t mainst = h->stream;
+  cudaStream_t side = forked ? h->side : mainst;
+  cudaStream_t upd = forked ? h->upd : mainst;
+  seg_status st;
   if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[L - 1], mainst), "event record");
   for (int l = L - 1; l >= 0; --l) {
     const LayerInfo& Ly = h->layers[l];
@@ -659,6 +669,56 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
   if (st != SEG_OK) return st;
   ++h->step;
   if (y_out && (st = copy_out(h, y_out, batch)) != SEG_OK) return st;
+  return SEG_OK;
+}
+
+// Recovery step (Section 5 of the paper): the left segment keeps training through the frozen right one.
+seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x, const int32_t* cls,
+                             int32_t batch, float* loss_out) {
+  if (!left || !right || !x || !cls) return SEG_ERR_INVALID_ARG;
+  if (batch < 1 || batch > left->max_batch || batch > right->max_batch) return SEG_ERR_SHAPE;
+  if (left->is_final || !right->is_final) return SEG_ERR_STATE;
+  if (left->widths[left->n_layers] != right->widths[0]) return SEG_ERR_SHAPE;
+  if (left->precision != right->precision || left->stream != right->stream) return SEG_ERR_UNSUPPORTED;
+  seg_handle* h = left;
+  seg_handle* r = right;
+  const int Ll = h->n_layers, Lr = r->n_layers;
+  cudaStream_t s = h->stream;
+  seg_status st;
+  {
+    Launch lc(h, K_COPY);
+    SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
+                                   h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2, s),
+            "input staging");
+  }
+  if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
+  if ((st = forward_layers(r, h->act[Ll], h->ld_act[Ll], batch)) != SEG_OK) return st;
+  {
+    Launch l(r, K_LOSS, s);
+    SEG_TRY(r, launch_softmax_ce_loss((const float*)r->act[Lr], r->ld_act[Lr], h->cls_stage, r->n_classes, batch,
+                                      r->last_relu ? 1 : 0, r->dzbuf[Lr - 1], r->act_dt, r->act_round, r->ld_act[Lr],
+                                      r->loss_partials, r->loss_counter, loss_out ? loss_out : r->loss_slot, s),
+            "softmax-CE loss");
+  }
+  // through the frozen right segment: dgrad only, down to its input, which is the left segment's output
+  for (int l = Lr - 1; l >= 0; --l) {
+    const LayerInfo& Ly = r->layers[l];
+    GemmDesc d{};
+    d.A = r->dzbuf[l]; d.a_sm = r->ld_act[l + 1]; d.a_sk = 1; d.a_dt = r->act_dt;
+    d.B = weights_op(r, l); d.b_sk = Ly.ldw; d.b_sn = 1; d.b_dt = r->op_dt;
+    d.M = batch; d.N = Ly.in; d.K = Ly.out; d.c_dt = r->act_dt; d.c_round = r->act_round;
+    if (l > 0) {
+      d.C = r->dzbuf[l - 1]; d.ldc = r->ld_act[l];
+      d.epi = EPI_MASK; d.mask = r->act[l]; d.ldmask = r->ld_act[l];
+    } else {
+      d.C = h->dzbuf[Ll - 1]; d.ldc = h->ld_act[Ll];
+      if (h->last_relu) { d.epi = EPI_MASK; d.mask = h->act[Ll]; d.ldmask = h->ld_act[Ll]; }
+      else d.epi = EPI_PLAIN;
+    }
+    if ((st = run_gemm(r, d, K_DGRAD, s)) != SEG_OK) return st;
+  }
+  if ((st = enqueue_backward(h, batch, !h->profile && h->fork_enabled)) != SEG_OK) return st;
+  ++h->step;
   return SEG_OK;
 }
 

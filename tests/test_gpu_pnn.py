@@ -42,3 +42,32 @@ def test_two_partition_training_matches_the_oracle(name, epochs, label_dist):
     assert np.mean(pred_g == pred_o) > 0.99              # argmax may differ only on near-ties
     for seg in gpu:
         seg.close()
+
+
+@pytest.mark.parametrize("precision,backend,tol", [("fp32", "auto", 1e-4), ("bf16", "tcgen05", 2e-2), ("tf32", "tcgen05", 2e-3)])
+def test_recovery_step_matches_the_oracle(precision, backend, tol):
+    """Section 5 (recovery epochs): the left segment trained through the frozen right segment."""
+    import torch
+    from paper_2403_11204_b200 import binding
+    from parity_util import batch_arrays, bits_equal
+    w = wl.WORKLOADS["tiny"]
+    batch = 200
+    gl, ol = make_pair([784, 256, 136], 47, False, precision, "momentum", 0.01, batch, segment_id=0, gemm_backend=backend)
+    gr, orr = make_pair([136, 72, 47], 47, True, precision, "momentum", 0.01, batch, segment_id=1, gemm_backend=backend)
+    x, cls = batch_arrays(w, batch, 784, precision=precision)
+    xt, ct = to_device(x, cls, precision)
+    right_before = [t.clone() for l in range(2) for t in gr.params(l)]
+    for step in range(2):
+        loss_t = torch.zeros(1, device="cuda")
+        binding.recovery_step(gl, gr, xt, ct, loss_t)
+        gl.poll()
+        loss_o = pnn.recovery_step(ol, orr, x, cls.astype(np.int64))
+        assert abs(float(loss_t.item()) - loss_o) <= tol * abs(loss_o)
+        for l in range(2):
+            dW, db = gl.grads(l)
+            assert rel_err(dW.cpu().numpy(), ol.dW[l]) <= tol and rel_err(db.cpu().numpy(), ol.db[l]) <= tol
+            W, b = gl.params(l)
+            assert rel_err(W.cpu().numpy(), ol.W[l]) <= tol and rel_err(b.cpu().numpy(), ol.b[l]) <= tol
+    right_after = [t for l in range(2) for t in gr.params(l)]
+    assert all(torch.equal(a, b) for a, b in zip(right_before, right_after))       # frozen: bit-identical
+    gl.close(); gr.close()

@@ -67,3 +67,26 @@ def test_three_partitions_use_one_label_set_per_cut():
     x, cls = data(40)
     losses, _ = pnn.train_partitioned(segs, x, cls, 8, [1, 1, 2])
     assert [len(l) for l in losses] == [5, 5, 10]
+
+
+def test_recovery_step_equals_end_to_end_gradients_of_the_joined_network():
+    """Section 5: the left part is trained through the frozen right part.  Its gradients must be the
+    joined network's own (already pinned by finite differences), the right part must not move, and
+    the update must be the left optimizer's."""
+    left, right = make_net()
+    x, cls = data(20)
+    whole = OracleSegment([12, 10, 8, 9, 4], 4, True, precision="fp64", optimizer="momentum", lr=0.05)
+    whole.W, whole.b = [w.copy() for w in left.W + right.W], [b.copy() for b in left.b + right.b]
+    loss_whole = whole.loss_and_grads(x, cls)
+    right_before = [p.copy() for p in right.W + right.b]
+    left_before = [p.copy() for p in left.W + left.b]
+    loss = pnn.recovery_step(left, right, x, cls)
+    assert abs(loss - loss_whole) < 1e-14
+    for l in range(2):
+        assert np.allclose(left.dW[l], whole.dW[l], rtol=1e-12, atol=1e-16)
+        assert np.allclose(left.db[l], whole.db[l], rtol=1e-12, atol=1e-16)
+    assert all(np.array_equal(a, b) for a, b in zip(right_before, right.W + right.b))
+    for p0, p1, g in zip(left_before, left.W + left.b, left.dW + left.db):
+        assert np.allclose(p1, p0 - 0.05 * g, rtol=1e-13, atol=1e-18)     # first momentum step = SGD step
+    losses = [pnn.recovery_step(left, right, x, cls) for _ in range(5)]
+    assert losses[-1] < loss                                               # recovery lowers the joined loss
