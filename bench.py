@@ -426,7 +426,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="paper_shaped", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--others", default="bf16_wide,gemm_large,multi_cut,tiny",
+    ap.add_argument("--others", default="bf16_wide,gemm_large,multi_cut,tiny,paper_net",
                     help="further workloads summarised in the same line ('' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--samples", type=int, default=0, help="size of the resident data set (0: the workload's own)")

@@ -128,6 +128,14 @@ SEG_API seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, fl
 SEG_API seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
                           float* loss_out, void* y_out);
 
+/* The step of the fully separate variant (Section 2, the flowchart in which middle
+ * partitions are trained with intermediate labels both as input and as target): the input
+ * of sample b is row cls[b] of sil_in, the [M][widths[0]] fp32 label matrix of the PREVIOUS
+ * cut (as seg_get_labels of the previous segment returns it); it is gathered on the device,
+ * no per-sample input tensor is materialised.  Everything else as seg_train_step.          */
+SEG_API seg_status seg_train_step_label_input(seg_handle* h, const float* sil_in, const int32_t* cls,
+                                              int32_t batch, float* loss_out);
+
 /* The same step for callers whose batch lives in HOST memory: copies x_host and cls_host
  * (host pointers; page-locked memory gives full copy speed) to device buffers the handle
  * owns (allocated at the first such call), runs seg_train_step, copies the loss back to

@@ -36,6 +36,7 @@ EXPORTS = {
     "seg_create": (c_int32, [POINTER(seg_config), POINTER(c_void_p)]),
     "seg_gen_labels": (c_int32, [c_void_p, c_uint64, c_int32, c_float]),
     "seg_train_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
+    "seg_train_step_label_input": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_train_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_float)]),
     "seg_forward": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_recovery_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
@@ -215,6 +216,14 @@ class Segment:
         self._check(self.lib.seg_train_step(self.h, _ptr(x), _ptr(cls), batch, _ptr(loss_out), _ptr(y_out)),
                     "seg_train_step")
         self.last_batch = batch
+
+    def train_step_label_input(self, sil_in, cls, loss_out=None):
+        """seg_train_step_label_input: the sample's input is row cls[b] of the previous cut's label matrix."""
+        assert sil_in.is_cuda and sil_in.is_contiguous() and sil_in.dtype == self._torch.float32
+        assert sil_in.shape == (self.n_classes, self.widths[0]) and cls.is_cuda and cls.dtype == self._torch.int32
+        self._check(self.lib.seg_train_step_label_input(self.h, _ptr(sil_in), _ptr(cls), cls.shape[0], _ptr(loss_out)),
+                    "seg_train_step_label_input")
+        self.last_batch = cls.shape[0]
 
     def train_step_host(self, x_host, cls_host):
         """x_host / cls_host: CPU tensors (pinned for speed).  Returns the loss as a float."""

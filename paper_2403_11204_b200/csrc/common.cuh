@@ -85,10 +85,12 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s);
 cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt,
                           int64_t ld_src, int rows, int cols, int round, cudaStream_t s);
 // the same copy plus an int32 vector copy (class indices) in one launch; when t is not null the
-// launch also advances the step counter: t += 1, bc = {1 - beta1^t, 1 - beta2^t}
+// launch also advances the step counter: t += 1, bc = {1 - beta1^t, 1 - beta2^t}; when gather_src is not
+// null, row r of the destination is row cls[r] of that fp32 [classes][cols] matrix instead of src's row r
 cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
-                                unsigned long long* t, float* bc, float beta1, float beta2, cudaStream_t s);
+                                unsigned long long* t, float* bc, float beta1, float beta2,
+                                const float* gather_src, cudaStream_t s);
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // Kernels of one stream are launched with programmatic stream serialisation: a kernel may become

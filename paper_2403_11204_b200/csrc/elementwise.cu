@@ -271,7 +271,7 @@ copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt
 __global__ void __launch_bounds__(256)
 stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows, int cols,
                     int round, int32_t* cls_dst, const int32_t* cls_src, unsigned long long* t, float* bc,
-                    float beta1, float beta2) {
+                    float beta1, float beta2, const float* gather_src) {
   pdl_wait();
   pdl_trigger();
   const int64_t total = (int64_t)rows * cols;
@@ -284,8 +284,10 @@ stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t 
   }
   for (int64_t e = tid; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = e / cols, c = e % cols;
-    const float v = apply_round(load_as_float(src, dt, r * ld_src + c), round);
-    store_from_float(dst, dt, r * ld_dst + c, v);
+    // gather_src: the input of sample r is row cls[r] of an fp32 label matrix (the fully separate variant)
+    const float raw = gather_src ? __ldg(gather_src + (int64_t)__ldg(cls_src + r) * cols + c)
+                                 : load_as_float(src, dt, r * ld_src + c);
+    store_from_float(dst, dt, r * ld_dst + c, apply_round(raw, round));
   }
   for (int64_t i = tid; i < rows; i += (int64_t)gridDim.x * blockDim.x) cls_dst[i] = cls_src[i];
 }
@@ -376,10 +378,11 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
 
 cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
-                                unsigned long long* t, float* bc, float beta1, float beta2, cudaStream_t s) {
+                                unsigned long long* t, float* bc, float beta1, float beta2,
+                                const float* gather_src, cudaStream_t s) {
   const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
   launch_k(stage_inputs_kernel, dim3(grid), dim3(256), 0, s, dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
-                                           beta1, beta2);
+                                           beta1, beta2, gather_src);
   return cudaGetLastError();
 }
 

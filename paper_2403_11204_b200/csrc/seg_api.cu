@@ -88,6 +88,7 @@ struct seg_handle {
     cudaKernelNodeParams stage_params{}, loss_params{};
     std::vector<void*> stage_args, loss_args;
     const void* cur_x = nullptr; const int32_t* cur_cls = nullptr; float* cur_loss = nullptr;   // now in the exec
+    const float* cur_gather = nullptr;
   };
   cudaGraphNode_t cap_stage_node = nullptr, cap_loss_node = nullptr;   // filled while capturing
   bool capturing = false;
@@ -477,7 +478,7 @@ static cudaGraphNode_t last_captured_node(seg_handle* h) {
 static seg_status enqueue_backward(seg_handle* h, int batch, bool forked);
 
 static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void* x, const int32_t* cls,
-                               float* loss_out) {
+                               float* loss_out, const float* gather) {
   const int L = h->n_layers;
   cudaStream_t mainst = h->stream;
   seg_status st;
@@ -488,7 +489,7 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   mainst), "input staging");
+                                   gather, mainst), "input staging");
   }
   if (h->capturing) h->cap_stage_node = last_captured_node(h);
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
@@ -581,7 +582,7 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
 }
 
 // Index of the caller-supplied pointers in the kernels' parameter lists (see elementwise.cu).
-static const int kStageArgCount = 14, kStageArgX = 3, kStageArgCls = 9;
+static const int kStageArgCount = 15, kStageArgX = 3, kStageArgCls = 9, kStageArgGather = 14;
 static int loss_arg_count(const seg_handle* h) { return h->is_final ? 12 : 13; }
 
 static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGraph_t graph) {
@@ -597,15 +598,16 @@ static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGr
 }
 
 static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const void* x, const int32_t* cls,
-                               float* loss_out) {
+                               float* loss_out, const float* gather) {
   float* loss_dst = loss_out ? loss_out : h->loss_slot;
-  if (x != g.cur_x || cls != g.cur_cls) {
+  if (x != g.cur_x || cls != g.cur_cls || gather != g.cur_gather) {
     g.stage_args[kStageArgX] = (void*)&x;
     g.stage_args[kStageArgCls] = (void*)&cls;
+    g.stage_args[kStageArgGather] = (void*)&gather;
     cudaKernelNodeParams sp = g.stage_params;
     sp.kernelParams = g.stage_args.data();
     SEG_TRY(h, cudaGraphExecKernelNodeSetParams(g.exec, g.stage_node, &sp), "graph parameter update");
-    g.cur_x = x; g.cur_cls = cls;
+    g.cur_x = x; g.cur_cls = cls; g.cur_gather = gather;
   }
   if (loss_dst != g.cur_loss) {
     g.loss_args[loss_arg_count(h) - 1] = (void*)&loss_dst;
@@ -619,20 +621,36 @@ static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const vo
   return SEG_OK;
 }
 
+static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
+                                  float* loss_out, void* y_out, const float* gather);
+
 seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
                           float* loss_out, void* y_out) {
   if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
+  return train_step_impl(h, x, cls, batch, loss_out, y_out, nullptr);
+}
+
+// Fully separate variant (Section 2, last flowchart): the segment's input is the intermediate label of the
+// previous cut, gathered by class inside the staging kernel.
+seg_status seg_train_step_label_input(seg_handle* h, const float* sil_in, const int32_t* cls, int32_t batch,
+                                      float* loss_out) {
+  if (!h || !sil_in || !cls) return SEG_ERR_INVALID_ARG;
+  return train_step_impl(h, nullptr, cls, batch, loss_out, nullptr, sil_in);
+}
+
+static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
+                                  float* loss_out, void* y_out, const float* gather) {
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   if (!h->is_final && !h->have_labels) return SEG_ERR_STATE;
   seg_status st = SEG_OK;
   if (h->profile || !h->graphs_enabled) {
-    st = enqueue_step(h, batch, !h->profile && h->fork_enabled, x, cls, loss_out);
+    st = enqueue_step(h, batch, !h->profile && h->fork_enabled, x, cls, loss_out, gather);
   } else {
     seg_handle::StepGraph& g = h->graphs[batch];
     if (g.exec != nullptr) {
-      st = replay_graph(h, g, x, cls, loss_out);
+      st = replay_graph(h, g, x, cls, loss_out, gather);
     } else if (g.eager_runs == 0) {
-      st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);   // first step at this batch size: eager (sets kernel attributes)
+      st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);   // first step at this batch size: eager (sets kernel attributes)
       g.eager_runs = 1;
     } else {
       const uint64_t before = h->launches;
@@ -640,16 +658,16 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
       if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         cudaGetLastError();
         h->graphs_enabled = false;
-        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);
+        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
       } else {
         h->capturing = true; h->cap_stage_node = nullptr; h->cap_loss_node = nullptr;
-        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);
+        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
         h->capturing = false;
         cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
         if (st == SEG_OK && e == cudaSuccess && graph != nullptr && adopt_captured_graph(h, g, graph)) {
           g.kernels = h->launches - before;
           h->launches = before;
-          st = replay_graph(h, g, x, cls, loss_out);
+          st = replay_graph(h, g, x, cls, loss_out, gather);
         } else {
           // capture did not work here: run eagerly from now on
           if (getenv("SEG_DEBUG"))
@@ -661,7 +679,7 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
           g.exec = nullptr;
           h->graphs_enabled = false;
           h->launches = before;
-          st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out);
+          st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
         }
       }
     }
@@ -688,8 +706,8 @@ seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x,
   {
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
-                                   h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2, s),
-            "input staging");
+                                   h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
+                                   nullptr, s), "input staging");
   }
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
   if ((st = forward_layers(r, h->act[Ll], h->ld_act[Ll], batch)) != SEG_OK) return st;

@@ -71,3 +71,37 @@ def test_recovery_step_matches_the_oracle(precision, backend, tol):
     right_after = [t for l in range(2) for t in gr.params(l)]
     assert all(torch.equal(a, b) for a, b in zip(right_before, right_after))       # frozen: bit-identical
     gl.close(); gr.close()
+
+
+@pytest.mark.parametrize("precision,backend,tol", [("fp32", "auto", 1e-4), ("bf16", "tcgen05", 2e-2)])
+def test_fully_separate_variant_label_rows_as_input(precision, backend, tol):
+    """Section 2, last flowchart: a middle partition trained with the previous cut's labels as input and
+    its own cut's labels as target; the input rows are gathered by class on the device."""
+    import torch
+    from oracle import rng as orng
+    from parity_util import compare_step, bits_equal
+    w = wl.WORKLOADS["tiny"]
+    m, batch = 47, 150
+    prev_labels = orng.gen_labels(wl.LABEL_SEED, 0, m, 136, orng.DIST_UNIFORM_KAPPA, 10.0)     # cut 0: 47 x 136
+    gpu, ora = make_pair([136, 200, 72], m, False, precision, "momentum", 0.01, batch, segment_id=1,
+                         gemm_backend=backend, label_dist="uniform_kappa")
+    cls = wl.class_indices(w, batch)
+    sil_t = torch.from_numpy(prev_labels).cuda()
+    ct = torch.from_numpy(cls).cuda()
+    for step in range(3):                                   # eager, captured, replayed
+        loss_t = torch.zeros(1, device="cuda")
+        gpu.train_step_label_input(sil_t, ct, loss_t)
+        gpu.poll()
+        loss_o = ora.train_step(prev_labels[cls], cls.astype(np.int64))
+        assert abs(float(loss_t.item()) - loss_o) <= tol * abs(loss_o)
+        for l in range(2):
+            dW, db = gpu.grads(l)
+            assert rel_err(dW.cpu().numpy(), ora.dW[l]) <= tol and rel_err(db.cpu().numpy(), ora.db[l]) <= tol
+            W, b = gpu.params(l)
+            assert rel_err(W.cpu().numpy(), ora.W[l]) <= tol
+    # an ordinary step on the same handle afterwards still reads the caller's x
+    x = prev_labels[cls]
+    if precision == "bf16":
+        x = wl.from_bf16_bits(wl.to_bf16_bits(x))
+    compare_step(gpu, ora, x, cls, precision, tol)
+    gpu.close()
