@@ -152,6 +152,10 @@ def test_argument_errors_and_state():
     with pytest.raises(SegError) as e:
         seg.train_step(torch.zeros(9, 16, device="cuda"), torch.zeros(9, dtype=torch.int32, device="cuda"))
     assert e.value.status == 2                             # batch > max_batch
+    empty = torch.zeros(0, 16, device="cuda")
+    with pytest.raises(SegError) as e:
+        seg.train_step(empty, torch.zeros(0, dtype=torch.int32, device="cuda"))
+    assert e.value.status in (1, 2)                        # an empty batch is refused (null pointer or shape), nothing is enqueued
     seg.train_step(x, c)
     seg.poll()
     cur, peak = seg.mem_bytes()
@@ -175,6 +179,13 @@ TC_CASES = [
     ([64, 128], False, "tf32", "sgd", 128),
     ([784, 320, 200, 72], False, "tf32", "adam", 300),
     ([72, 136, 264, 47], True, "tf32", "adam", 129),
+    # the paper's own partitions (Section 3) on tensor cores: widths 80 / 60 / 47 are not multiples of 8 elements
+    ([784, 80, 60], False, "bf16", "momentum", 1410),
+    ([60, 60, 60, 47], True, "bf16", "momentum", 1410),
+    ([784, 80, 60], False, "tf32", "momentum", 1410),
+    ([60, 60, 60, 47], True, "tf32", "momentum", 1410),
+    ([33, 17, 9], False, "bf16", "sgd", 5),                 # everything smaller than one tile, odd widths
+    ([8, 8], False, "tf32", "sgd", 1),                      # a single sample
 ]
 
 
@@ -184,7 +195,7 @@ def test_single_step_tensor_core_backend(widths, final, precision, optimizer, ba
     gpu, ora = make_pair(widths, 47, final, precision, optimizer, 1e-3, batch, gemm_backend="tcgen05")
     x, cls = batch_arrays(w, batch, widths[0], precision=precision)
     compare_step(gpu, ora, x, cls, precision, TOL[precision])
-    x2, cls2 = batch_arrays(w, batch - 1, widths[0], seed=5, precision=precision)
+    x2, cls2 = batch_arrays(w, max(batch - 1, 1), widths[0], seed=5, precision=precision)
     if optimizer == "adam":
         sync_from_oracle(gpu, ora)
     compare_step(gpu, ora, x2, cls2, precision, TOL[precision])      # smaller batch on the same handle
