@@ -22,6 +22,16 @@
  *   - Nothing is thrown across this boundary and nothing aborts the process.
  *   - A handle is not thread-safe; different handles may be used from different
  *     threads and on different streams concurrently.
+ *
+ * Diagnostic environment switches, read when a handle is created (first handle of the
+ * process for the kernel-selection ones); all default to off / automatic:
+ *   SEG_NO_GRAPH=1        launch every kernel eagerly instead of replaying a captured step
+ *   SEG_NO_FORK=1         run the three branches of a step on one stream
+ *   SEG_NO_PDL=1          ordinary launches instead of programmatic dependent launches
+ *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
+ *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
+ *   SEG_PAIR_MIN_TILES=n  use CTA pairs from n tiles of 256 x 256 on (default 96)
+ *   SEG_DEBUG=1           report on stderr when a step could not be captured into a graph
  */
 #ifndef SEG_H_
 #define SEG_H_
