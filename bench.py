@@ -329,12 +329,10 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
                 k["ms"] += tot
                 if name in ("fwd_gemm", "dgrad_gemm", "wgrad_gemm"):
                     k["flops"] += work[name] * steps
-                elif name == "update":
-                    k["bytes"] += work["update_bytes"] * steps
+                elif name == "update":          # the update launch also reads dZ for the bias gradient
+                    k["bytes"] += (work["update_bytes"] + work["bias_grad_bytes"]) * steps
                 elif name == "loss":
                     k["bytes"] += work["loss_bytes"] * steps
-                elif name == "bias_grad":
-                    k["bytes"] += work["bias_grad_bytes"] * steps
             seg.profile(False)
         out["kernels"] = {n: {"launches": v["launches"], "ms_total": round(v["ms"], 4),
                               "avg_us": round(1e3 * v["ms"] / max(v["launches"], 1), 3)} for n, v in kinds.items()}

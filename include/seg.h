@@ -26,7 +26,7 @@
  * Diagnostic environment switches, read when a handle is created (first handle of the
  * process for the kernel-selection ones); all default to off / automatic:
  *   SEG_NO_GRAPH=1        launch every kernel eagerly instead of replaying a captured step
- *   SEG_NO_FORK=1         run the three branches of a step on one stream
+ *   SEG_NO_FORK=1         run every branch of a step on one stream
  *   SEG_NO_PDL=1          ordinary launches instead of programmatic dependent launches
  *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
  *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
@@ -236,7 +236,8 @@ SEG_API seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms);
  * bracketed by CUDA events on the handle's stream.  seg_profile_get synchronises and
  * returns, for one kernel kind, the number of launches and their summed device time
  * since profiling was enabled; kinds: 0 forward product, 1 dgrad product, 2 wgrad
- * product, 3 loss, 4 bias gradient, 5 optimizer update, 6 copies / staging.  count and
+ * product, 3 loss, 4 unused (always 0 launches), 5 optimizer update (forms the bias gradient
+ * too), 6 copies / staging.  count and
  * total_ms are host pointers.                                                            */
 SEG_API seg_status seg_profile_enable(seg_handle* h, int32_t on);
 SEG_API seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms);

@@ -20,7 +20,8 @@ PRECISIONS = {"fp32": SEG_FP32, "tf32": SEG_TF32, "bf16": SEG_BF16}
 OPTIMIZERS = {"sgd": SEG_SGD, "momentum": SEG_SGD_MOMENTUM, "adam": SEG_ADAM}
 LABEL_DISTS = {"uniform_kappa": SEG_LABEL_UNIFORM_KAPPA, "normal": SEG_LABEL_NORMAL}
 BACKENDS = {"auto": SEG_GEMM_AUTO, "simt": SEG_GEMM_SIMT, "tcgen05": SEG_GEMM_TCGEN05}
-KERNEL_KINDS = ["fwd_gemm", "dgrad_gemm", "wgrad_gemm", "loss", "bias_grad", "update", "copy"]
+# kind numbers of seg_profile_get (4 is unused: the update launch forms the bias gradient)
+KERNEL_KINDS = {0: "fwd_gemm", 1: "dgrad_gemm", 2: "wgrad_gemm", 3: "loss", 5: "update", 6: "copy"}
 
 
 class seg_config(Structure):
@@ -343,7 +344,7 @@ class Segment:
 
     def profile_read(self):
         out = {}
-        for k, name in enumerate(KERNEL_KINDS):
+        for k, name in KERNEL_KINDS.items():
             n, ms = c_uint64(), c_float()
             self._check(self.lib.seg_profile_get(self.h, k, byref(n), byref(ms)))
             out[name] = (n.value, ms.value)

@@ -63,18 +63,22 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
                                    cudaStream_t s);
 int loss_max_partials();
 
-// db[n] = sum_b dZ[b][n], deterministic
-cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, int n, float* db,
-                             float* partials, unsigned int* counters, cudaStream_t s);
-int bias_grad_partial_floats(int batch, int n);
-int bias_grad_counters(int n);
-
+// One layer's update.  p, g, s1, s2, p_op point at the layer's weight tensor in the flat ranges; n
+// elements from there are streamed (the weight tensor with its zero padding).  When dz is not null
+// the launch also forms the bias gradient g_bias[c] = sum_b dz[b][c], c < n_bias, and updates the
+// n_bias bias elements that start bias_off elements after p.
 struct UpdateArgs {
   float* p; const float* g; float* s1; float* s2;
   void* p_op;          // reduced-precision operand copy (may be null)
   int op_dt;           // DType of p_op
   int op_round;        // Round for p_op
   int64_t n;
+  const void* dz;      // [batch][ld_dz] of dz_dt: dZ of this layer (may be null: no bias part)
+  int dz_dt;
+  int64_t ld_dz;
+  int batch, n_bias;
+  int64_t bias_off;
+  float* g_bias;       // [n_bias]: receives the bias gradient
   int optimizer;
   float lr, momentum, beta1, beta2, eps;
   const float* bc;     // device: {1-b1^t, 1-b2^t}, Adam's bias corrections for this step

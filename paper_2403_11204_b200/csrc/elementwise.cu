@@ -1,6 +1,6 @@
 // Streaming kernels of the segment step: the two losses (Section 2: intermediate-label
-// regression for a non-final segment, class labels for the final one), the bias gradient,
-// the fused optimizer update (Section 3: SGD with momentum; plain SGD and Adam as well) and
+// regression for a non-final segment, class labels for the final one), the optimizer update
+// with the bias gradient formed in the same launch (Section 3: SGD with momentum; plain SGD and Adam as well) and
 // pitch/dtype conversion copies.  All of them are HBM-bound; none uses tensor cores.
 #include "common.cuh"
 
@@ -136,106 +136,95 @@ softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* _
   finish_loss(bt, partials, counter, loss_out, inv_b, red);
 }
 
-// db[n] = sum_b dZ[b][n].  Grid (column strips of 32, row chunks): every block sums its rows with
-// 8 row lanes, writes one partial per column to scratch[chunk][n]; the last block of a strip to
-// finish adds the chunk partials in chunk order (fixed order: bit-reproducible) and resets the
-// strip's arrival counter.
-constexpr int kBiasRowsPerChunk = 128;
-template <typename T>
-__global__ void __launch_bounds__(256)
-bias_grad_kernel(const T* __restrict__ dz, int64_t ld, int batch, int n, float* __restrict__ db,
-                 float* __restrict__ scratch, unsigned int* __restrict__ counters) {
-  pdl_wait();
-  pdl_trigger();
-  __shared__ float part[8][33];
-  __shared__ bool is_last;
-  const int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
-  const int col = blockIdx.x * 32 + lane;
-  const int r0 = blockIdx.y * kBiasRowsPerChunk;
-  const int r1 = (gridDim.y == 1) ? batch : min(batch, r0 + kBiasRowsPerChunk);
-  float acc = 0.f;
-  if (col < n) {
-#pragma unroll 4
-    for (int b = r0 + rl; b < r1; b += 8) {
-      if constexpr (sizeof(T) == 2) acc += __bfloat162float(dz[(int64_t)b * ld + col]);
-      else acc += dz[(int64_t)b * ld + col];
-    }
-  }
-  part[rl][lane] = acc;
-  __syncthreads();
-  if (rl == 0) {
-    float s = 0.f;
-#pragma unroll
-    for (int r = 0; r < 8; ++r) s += part[r][lane];
-    if (gridDim.y == 1) {
-      if (col < n) db[col] = s;
-    } else if (col < n) {
-      scratch[(int64_t)blockIdx.y * n + col] = s;
-    }
-  }
-  if (gridDim.y == 1) return;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(counters + blockIdx.x, 1u) == gridDim.y - 1);
-  __syncthreads();
-  if (is_last && rl == 0) {
-    __threadfence();
-    if (col < n) {
-      float s = 0.f;
-      for (unsigned int c = 0; c < gridDim.y; ++c) s += __ldcg(scratch + (int64_t)c * n + col);
-      db[col] = s;
-    }
-    if (lane == 0) counters[blockIdx.x] = 0u;
+// One optimizer step on one element (Section 3: SGD with momentum; plain SGD and Adam as well).
+template <int OPT>
+__device__ __forceinline__ void opt_step(float& p, float g, float& m, float& v, const UpdateArgs& u,
+                                         float inv_bc1, float inv_bc2) {
+  if constexpr (OPT == SEG_SGD) {
+    p = p - u.lr * g;
+  } else if constexpr (OPT == SEG_SGD_MOMENTUM) {
+    m = u.momentum * m + g;
+    p = p - u.lr * m;
+  } else {
+    m = u.beta1 * m + (1.0f - u.beta1) * g;
+    v = u.beta2 * v + (1.0f - u.beta2) * g * g;
+    const float mhat = m * inv_bc1;
+    const float vhat = v * inv_bc2;
+    p = p - u.lr * mhat / (sqrtf(vhat) + u.eps);
   }
 }
 
-// One pass over the flat parameter range of a segment: parameters, gradients and optimizer
-// state share one layout, so a single launch updates every tensor and refreshes the
-// reduced-precision operand copy.
+// The update of one layer in one launch.  Parameters, gradients and optimizer state share one flat
+// layout [W | b]:
+//   blocks [0, bias_blocks): each forms the bias gradient of 32 columns, db[n] = sum_b dZ[b][n]
+//     (8 row lanes per column, then the lanes in index order: one fixed order, bit-reproducible),
+//     stores it and applies the optimizer to those bias elements;
+//   the other blocks stream over the weight range, whose gradient the weight-gradient product wrote.
+// Both parts refresh the reduced-precision operand copy.
 template <int OPT, int OPDT>
 __global__ void __launch_bounds__(256)
-update_kernel(UpdateArgs u) {
+update_kernel(UpdateArgs u, int bias_blocks) {
   pdl_wait();
   pdl_trigger();
+  float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
+  if constexpr (OPT == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(u.bc); inv_bc2 = 1.0f / __ldg(u.bc + 1); }
+  if ((int)blockIdx.x < bias_blocks) {
+    __shared__ float part[8][33];
+    const int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
+    const int col = blockIdx.x * 32 + lane;
+    float acc = 0.f;
+    if (col < u.n_bias) {
+      if (u.dz_dt == DT_BF16) {
+        const __nv_bfloat16* dz = reinterpret_cast<const __nv_bfloat16*>(u.dz);
+#pragma unroll 8
+        for (int b = rl; b < u.batch; b += 8) acc += __bfloat162float(dz[(int64_t)b * u.ld_dz + col]);
+      } else {
+        const float* dz = reinterpret_cast<const float*>(u.dz);
+#pragma unroll 8
+        for (int b = rl; b < u.batch; b += 8) acc += dz[(int64_t)b * u.ld_dz + col];
+      }
+    }
+    part[rl][lane] = acc;
+    __syncthreads();
+    if (rl == 0 && col < u.n_bias) {
+      float g = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) g += part[r][lane];
+      const int64_t i = u.bias_off + col;
+      u.g_bias[col] = g;
+      float p = u.p[i], m = 0.f, v = 0.f;
+      if constexpr (OPT != SEG_SGD) m = u.s1[i];
+      if constexpr (OPT == SEG_ADAM) v = u.s2[i];
+      opt_step<OPT>(p, g, m, v, u, inv_bc1, inv_bc2);
+      if constexpr (OPT != SEG_SGD) u.s1[i] = m;
+      if constexpr (OPT == SEG_ADAM) u.s2[i] = v;
+      u.p[i] = p;
+      if constexpr (OPDT == DT_BF16) {
+        reinterpret_cast<__nv_bfloat16*>(u.p_op)[i] = __float2bfloat16_rn(p);
+      } else {
+        if (u.p_op != nullptr) reinterpret_cast<float*>(u.p_op)[i] = apply_round(p, u.op_round);
+      }
+    }
+    return;
+  }
   const int64_t n4 = u.n >> 2;
   float4* __restrict__ p4 = reinterpret_cast<float4*>(u.p);
   const float4* __restrict__ g4 = reinterpret_cast<const float4*>(u.g);
   float4* __restrict__ s14 = reinterpret_cast<float4*>(u.s1);
   float4* __restrict__ s24 = reinterpret_cast<float4*>(u.s2);
-  float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
-  if constexpr (OPT == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(u.bc); inv_bc2 = 1.0f / __ldg(u.bc + 1); }
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4;
-       i += (int64_t)gridDim.x * blockDim.x) {
-    float4 p = p4[i];
+  const int64_t stride = (int64_t)(gridDim.x - bias_blocks) * blockDim.x;
+  for (int64_t i = (int64_t)(blockIdx.x - bias_blocks) * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    const float4 p = p4[i];
     const float4 g = g4[i];
     float pv[4] = {p.x, p.y, p.z, p.w};
     const float gv[4] = {g.x, g.y, g.z, g.w};
-    if constexpr (OPT == SEG_SGD) {
+    float mv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (OPT != SEG_SGD) { const float4 m = s14[i]; mv[0] = m.x; mv[1] = m.y; mv[2] = m.z; mv[3] = m.w; }
+    if constexpr (OPT == SEG_ADAM) { const float4 v = s24[i]; vv[0] = v.x; vv[1] = v.y; vv[2] = v.z; vv[3] = v.w; }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) pv[k] = pv[k] - u.lr * gv[k];
-    } else if constexpr (OPT == SEG_SGD_MOMENTUM) {
-      float4 m = s14[i];
-      float mv[4] = {m.x, m.y, m.z, m.w};
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        mv[k] = u.momentum * mv[k] + gv[k];
-        pv[k] = pv[k] - u.lr * mv[k];
-      }
-      s14[i] = make_float4(mv[0], mv[1], mv[2], mv[3]);
-    } else {
-      float4 m = s14[i], v = s24[i];
-      float mv[4] = {m.x, m.y, m.z, m.w}, vv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        mv[k] = u.beta1 * mv[k] + (1.0f - u.beta1) * gv[k];
-        vv[k] = u.beta2 * vv[k] + (1.0f - u.beta2) * gv[k] * gv[k];
-        const float mhat = mv[k] * inv_bc1;
-        const float vhat = vv[k] * inv_bc2;
-        pv[k] = pv[k] - u.lr * mhat / (sqrtf(vhat) + u.eps);
-      }
-      s14[i] = make_float4(mv[0], mv[1], mv[2], mv[3]);
-      s24[i] = make_float4(vv[0], vv[1], vv[2], vv[3]);
-    }
+    for (int k = 0; k < 4; ++k) opt_step<OPT>(pv[k], gv[k], mv[k], vv[k], u, inv_bc1, inv_bc2);
+    if constexpr (OPT != SEG_SGD) s14[i] = make_float4(mv[0], mv[1], mv[2], mv[3]);
+    if constexpr (OPT == SEG_ADAM) s24[i] = make_float4(vv[0], vv[1], vv[2], vv[3]);
     p4[i] = make_float4(pv[0], pv[1], pv[2], pv[3]);
     if constexpr (OPDT == DT_BF16) {
       __nv_bfloat162 lo = __floats2bfloat162_rn(pv[0], pv[1]);
@@ -339,33 +328,15 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
   return cudaGetLastError();
 }
 
-// scratch: `partials` holds [chunks][n] floats, `counters` one arrival counter per strip of 32 columns
-// (zero-initialised once; the kernel leaves them at zero).  With partials == nullptr one block per
-// strip walks all rows.
-int bias_grad_partial_floats(int batch, int n) {
-  return ((batch + kBiasRowsPerChunk - 1) / kBiasRowsPerChunk) * n;
-}
-int bias_grad_counters(int n) { return (n + 31) / 32; }
-
-cudaError_t launch_bias_grad(const void* dz, int dz_dt, int64_t ld, int batch, int n, float* db,
-                             float* partials, unsigned int* counters, cudaStream_t s) {
-  const int chunks = (batch + kBiasRowsPerChunk - 1) / kBiasRowsPerChunk;
-  dim3 grid((n + 31) / 32, (partials == nullptr || counters == nullptr) ? 1 : chunks);
-  if (dz_dt == DT_BF16)
-    launch_k(bias_grad_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, s, (const __nv_bfloat16*)dz, ld, batch, n, db, partials, counters);
-  else
-    launch_k(bias_grad_kernel<float>, dim3(grid), dim3(256), 0, s, (const float*)dz, ld, batch, n, db, partials, counters);
-  return cudaGetLastError();
-}
-
 cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
-  if (u.n == 0) return cudaSuccess;
   if (u.n & 3) return cudaErrorInvalidValue;
-  const int grid = grid_for(u.n >> 2, 256, 148 * 8);
+  const int bias_blocks = (u.dz != nullptr && u.n_bias > 0) ? (u.n_bias + 31) / 32 : 0;
+  if (u.n == 0 && bias_blocks == 0) return cudaSuccess;
+  const int grid = bias_blocks + (u.n > 0 ? grid_for(u.n >> 2, 256, 148 * 8) : 0);
   const bool bf = (u.p_op != nullptr && u.op_dt == DT_BF16);
 #define SEGK_UPD(OPT)                                                      \
-  if (bf) launch_k(update_kernel<OPT, DT_BF16>, dim3(grid), dim3(256), 0, s, u);             \
-  else launch_k(update_kernel<OPT, DT_F32>, dim3(grid), dim3(256), 0, s, u)
+  if (bf) launch_k(update_kernel<OPT, DT_BF16>, dim3(grid), dim3(256), 0, s, u, bias_blocks);             \
+  else launch_k(update_kernel<OPT, DT_F32>, dim3(grid), dim3(256), 0, s, u, bias_blocks)
   switch (u.optimizer) {
     case SEG_SGD: SEGK_UPD(SEG_SGD); break;
     case SEG_SGD_MOMENTUM: SEGK_UPD(SEG_SGD_MOMENTUM); break;

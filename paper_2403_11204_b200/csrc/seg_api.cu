@@ -11,12 +11,13 @@
 //                      branch reads dZ_l while the main branch already produces dZ_{l-1}).
 //   sil              : [M][N_P] fp32 intermediate labels (Eq. 1).
 //
-// One training step is a three-branch dependency graph.  Main branch: forward products, loss, then
-// the dgrad chain.  Gradient branch: per layer the bias gradient and the weight-gradient product
-// (they need dZ_l only).  Update branch: per layer the optimizer update, which waits for that
-// layer's gradients and for its dgrad (the last reader of the old weights).  The HBM-bound updates
-// thereby run beside the tensor-core products of the layers below.  After one eager run per batch size the step is
-// captured into a CUDA graph and replayed; the caller's x / cls are first copied into
+// One training step is a dependency graph with one branch per layer.  Main branch: input staging,
+// forward products, loss, the dgrad chain, then layer 0's weight gradient and update.  Branch of
+// layer l >= 1: the weight-gradient product as soon as dZ_l exists, then the update of W_l and b_l
+// (the same launch forms the bias gradient), which also waits for dgrad(l), the last reader of the
+// old weights.  The upper layers' HBM-bound updates thereby run beside the tensor-core products of
+// the layers below, and only two kernels follow the last dgrad.  After one eager run per batch size
+// the step is captured into a CUDA graph and replayed; the caller's x / cls are first copied into
 // fixed staging buffers so that the graph never changes.
 #include <math.h>
 #include <stdio.h>
@@ -42,7 +43,7 @@ struct LayerInfo {
   int64_t w_off, b_off;  // element offsets into the flat ranges
 };
 
-enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_BIAS, K_UPDATE, K_COPY, K_COUNT };
+enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_UNUSED4, K_UPDATE, K_COPY, K_COUNT };   // values are part of the ABI
 
 int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 
@@ -71,12 +72,9 @@ struct seg_handle {
   float* loss_slot = nullptr;
   unsigned long long* step_dev = nullptr;
   float* bc_dev = nullptr;
-  float* bias_scratch = nullptr;
-  unsigned int* bias_counters = nullptr;
-  cudaStream_t side = nullptr, upd = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_join_upd = nullptr;
-  std::vector<cudaEvent_t> ev_dz;  // ev_dz[l]: dZ_l is complete (main branch)
-  std::vector<cudaEvent_t> ev_wg;  // ev_wg[l]: dW_l and db_l are complete (gradient branch)
+  std::vector<cudaStream_t> lstream;  // lstream[l], l >= 1: the branch of layer l (weight gradient, then update)
+  std::vector<cudaEvent_t> ev_dz;     // ev_dz[l]: dZ_l is complete (main branch)
+  std::vector<cudaEvent_t> ev_done;   // ev_done[l], l >= 1: layer l's branch is complete
   // A captured step.  The caller's pointers enter the graph in two kernel nodes only (input staging:
   // x and cls; loss: loss_out); their parameters are rewritten before every replay.
   struct StepGraph {
@@ -366,25 +364,14 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   if ((st = dev_alloc(h, &h->loss_slot, 1, true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->step_dev, 1, true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->bc_dev, 2, true)) != SEG_OK) return bail(st);
-  {
-    int floats = 0, counters = 0;
-    for (int l = 0; l < h->n_layers; ++l) {
-      floats = std::max(floats, bias_grad_partial_floats(h->max_batch, h->widths[l + 1]));
-      counters = std::max(counters, bias_grad_counters(h->widths[l + 1]));
-    }
-    if ((st = dev_alloc(h, &h->bias_scratch, floats, true)) != SEG_OK) return bail(st);
-    if ((st = dev_alloc(h, &h->bias_counters, counters, true)) != SEG_OK) return bail(st);
-  }
-  if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&h->upd, cudaStreamNonBlocking) != cudaSuccess) return bail(SEG_ERR_CUDA);
-  if (cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_join_upd, cudaEventDisableTiming) != cudaSuccess) return bail(SEG_ERR_CUDA);
+  h->lstream.assign(h->n_layers, nullptr);
   h->ev_dz.assign(h->n_layers, nullptr);
-  h->ev_wg.assign(h->n_layers, nullptr);
-  for (int l = 0; l < h->n_layers; ++l)
+  h->ev_done.assign(h->n_layers, nullptr);
+  for (int l = 0; l < h->n_layers; ++l) {
+    if (l > 0 && cudaStreamCreateWithFlags(&h->lstream[l], cudaStreamNonBlocking) != cudaSuccess) return bail(SEG_ERR_CUDA);
     if (cudaEventCreateWithFlags(&h->ev_dz[l], cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_wg[l], cudaEventDisableTiming) != cudaSuccess) return bail(SEG_ERR_CUDA);
+        cudaEventCreateWithFlags(&h->ev_done[l], cudaEventDisableTiming) != cudaSuccess) return bail(SEG_ERR_CUDA);
+  }
   {
     const char* env = getenv("SEG_NO_GRAPH");
     if (env && env[0] == '1') h->graphs_enabled = false;
@@ -419,19 +406,14 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
 seg_status seg_destroy(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
   cudaStreamSynchronize(h->stream);
-  if (h->side) cudaStreamSynchronize(h->side);
-  if (h->upd) cudaStreamSynchronize(h->upd);
+  for (cudaStream_t ls : h->lstream) if (ls) cudaStreamSynchronize(ls);
   for (auto& kv : h->graphs) {
     if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
     if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
   }
   for (cudaEvent_t e : h->ev_dz) if (e) cudaEventDestroy(e);
-  for (cudaEvent_t e : h->ev_wg) if (e) cudaEventDestroy(e);
-  if (h->ev_join_upd) cudaEventDestroy(h->ev_join_upd);
-  if (h->upd) cudaStreamDestroy(h->upd);
-  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-  if (h->ev_join) cudaEventDestroy(h->ev_join);
-  if (h->side) cudaStreamDestroy(h->side);
+  for (cudaEvent_t e : h->ev_done) if (e) cudaEventDestroy(e);
+  for (cudaStream_t ls : h->lstream) if (ls) cudaStreamDestroy(ls);
   for (void* p : h->allocations) cudaFree(p);
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->ev_start) cudaEventDestroy(h->ev_start);
@@ -511,20 +493,25 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
 }
 
 // Backward pass and update of every layer, starting from dZ of the last layer in dzbuf[L-1].
+// The main branch carries the dgrad chain and then layer 0's weight gradient and update, all linked
+// by programmatic dependent launches.  Every layer l >= 1 has a branch of its own: its weight
+// gradient starts as soon as dZ_l exists, its update (which also forms the bias gradient) follows
+// once dgrad(l), the last reader of the old W_l, is done.  The branches of the upper layers thereby
+// finish beside the dgrad chain, and what is left after the last dgrad is two kernels.
 static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
   const int L = h->n_layers;
   cudaStream_t mainst = h->stream;
-  cudaStream_t side = forked ? h->side : mainst;
-  cudaStream_t upd = forked ? h->upd : mainst;
   seg_status st;
-  if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[L - 1], mainst), "event record");
+  if (forked && L > 1) SEG_TRY(h, cudaEventRecord(h->ev_dz[L - 1], mainst), "event record");
   for (int l = L - 1; l >= 0; --l) {
     const LayerInfo& Ly = h->layers[l];
     const int64_t ld_dz = h->ld_act[l + 1];
     const void* dz_l = h->dzbuf[l];
     const void* a_prev = (l == 0) ? h->x_stage : h->act[l];
     const int64_t ld_prev = h->ld_act[l];
-    // main branch first: dgrad of layer l, the last reader of the old W_l
+    const bool branch = forked && l > 0;
+    cudaStream_t ls = branch ? h->lstream[l] : mainst;
+    // main branch first: dgrad of layer l
     if (l > 0) {
       GemmDesc d{};
       d.A = dz_l; d.a_sm = ld_dz; d.a_sk = 1; d.a_dt = h->act_dt;
@@ -535,49 +522,35 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
       if ((st = run_gemm(h, d, K_DGRAD, mainst)) != SEG_OK) return st;
       if (forked) SEG_TRY(h, cudaEventRecord(h->ev_dz[l - 1], mainst), "event record");
     }
-    // gradient branch: weight gradient of layer l (needs dZ_l)
-    if (forked) SEG_TRY(h, cudaStreamWaitEvent(side, h->ev_dz[l], 0), "stream wait");
-    const int64_t lo = Ly.w_off;
-    const int64_t hi = (l + 1 < L) ? h->layers[l + 1].w_off : h->n_flat;
+    // weight gradient of layer l (needs dZ_l)
+    if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l], 0), "stream wait");
     GemmDesc w{};
     w.A = dz_l; w.a_sm = 1; w.a_sk = ld_dz; w.a_dt = h->act_dt;
     w.B = a_prev; w.b_sk = ld_prev; w.b_sn = 1; w.b_dt = h->act_dt;
     w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
     w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
-    if ((st = run_gemm(h, w, K_WGRAD, side)) != SEG_OK) return st;
-    if (forked) SEG_TRY(h, cudaEventRecord(h->ev_wg[l], side), "event record");
-    // update branch: the bias gradient (needs dZ_l only, so it runs beside the weight-gradient product),
-    // then the update of layer l's tensors (W_l and b_l are adjacent in the flat range)
-    if (forked) SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_dz[l], 0), "stream wait");
-    {
-      Launch lb(h, K_BIAS, upd);
-      SEG_TRY(h, launch_bias_grad(dz_l, h->act_dt, ld_dz, batch, Ly.out, h->grads + Ly.b_off, h->bias_scratch,
-                                  h->bias_counters, upd), "bias gradient");
-    }
-    if (forked) {
-      SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_wg[l], 0), "stream wait");
-      if (l > 0) SEG_TRY(h, cudaStreamWaitEvent(upd, h->ev_dz[l - 1], 0), "stream wait");   // dgrad(l) done
-    }
-    const int64_t ulo = lo;
+    if ((st = run_gemm(h, w, K_WGRAD, ls)) != SEG_OK) return st;
+    // update of W_l and b_l (adjacent in the flat range) once dgrad(l) no longer reads the old W_l
+    if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
+    const int64_t lo = Ly.w_off;
     UpdateArgs u{};
-    u.p = h->params + ulo; u.g = h->grads + ulo;
-    u.s1 = h->state1 ? h->state1 + ulo : nullptr; u.s2 = h->state2 ? h->state2 + ulo : nullptr;
-    u.p_op = h->params_op ? (void*)(reinterpret_cast<char*>(h->params_op) + ulo * elem_size(h->op_dt)) : nullptr;
+    u.p = h->params + lo; u.g = h->grads + lo;
+    u.s1 = h->state1 ? h->state1 + lo : nullptr; u.s2 = h->state2 ? h->state2 + lo : nullptr;
+    u.p_op = h->params_op ? (void*)(reinterpret_cast<char*>(h->params_op) + lo * elem_size(h->op_dt)) : nullptr;
     u.op_dt = h->op_dt; u.op_round = h->op_round;
-    u.n = hi - ulo; u.optimizer = h->optimizer;
+    u.n = Ly.b_off - lo; u.optimizer = h->optimizer;
+    u.dz = dz_l; u.dz_dt = h->act_dt; u.ld_dz = ld_dz; u.batch = batch; u.n_bias = Ly.out;
+    u.bias_off = Ly.b_off - lo; u.g_bias = h->grads + Ly.b_off;
     u.lr = h->lr; u.momentum = h->momentum; u.beta1 = h->beta1; u.beta2 = h->beta2; u.eps = h->eps;
     u.bc = h->bc_dev;
     {
-      Launch lu(h, K_UPDATE, upd);
-      SEG_TRY(h, launch_update(u, upd), "optimizer update");
+      Launch lu(h, K_UPDATE, ls);
+      SEG_TRY(h, launch_update(u, ls), "optimizer update");
     }
+    if (branch) SEG_TRY(h, cudaEventRecord(h->ev_done[l], ls), "event record");
   }
-  if (forked) {
-    SEG_TRY(h, cudaEventRecord(h->ev_join, side), "event record");
-    SEG_TRY(h, cudaEventRecord(h->ev_join_upd, upd), "event record");
-    SEG_TRY(h, cudaStreamWaitEvent(mainst, h->ev_join, 0), "stream wait");
-    SEG_TRY(h, cudaStreamWaitEvent(mainst, h->ev_join_upd, 0), "stream wait");
-  }
+  if (forked)
+    for (int l = 1; l < L; ++l) SEG_TRY(h, cudaStreamWaitEvent(mainst, h->ev_done[l], 0), "stream wait");
   return SEG_OK;
 }
 
