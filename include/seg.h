@@ -30,7 +30,8 @@
  *   SEG_NO_PDL=1          ordinary launches instead of programmatic dependent launches
  *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
  *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
- *   SEG_PAIR_MIN_TILES=n  use CTA pairs from n tiles of 256 x 256 on (default 96)
+ *   SEG_PAIR_MIN_TILES=n  use CTA pairs exactly when a product has n or more tiles of 256 x 256
+ *                         (default: a cost model of the main loop chooses)
  *   SEG_DEBUG=1           report on stderr when a step could not be captured into a graph
  */
 #ifndef SEG_H_

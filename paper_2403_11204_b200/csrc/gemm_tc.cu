@@ -182,13 +182,16 @@ struct SmemLayout {
   static constexpr int TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
 };
 
-// Epilogue for up to 32 consecutive columns of one row.  Columns are handled in groups of 8 with
-// 16-byte accesses when the group count is whole and the row segment is 16-byte aligned (every
-// lane touches its own row, so wide accesses are what keeps the number of memory wavefronts down);
-// ragged or unaligned segments fall back to scalar accesses.
-__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], int row, int col0,
-                                               int n_total) {
+// Side inputs of the epilogue for up to 32 consecutive columns of one row: the bias values (forward)
+// or the stored activations that give the ReLU mask (dgrad; bf16 activations packed two per word).
+// They do not depend on the accumulator, so they are fetched before it is waited for and their
+// global-memory latency is off the critical path.
+struct EpiSide { uint32_t w[32]; };
+
+__device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide& s, int row, bool row_ok,
+                                                  int col0, int n_total) {
   const int n_valid = min(32, n_total - col0);
+  if (n_valid <= 0) return;
   const bool whole = (n_valid & 7) == 0;
   if (e.epi == EPI_BIAS_ACT) {
     const float* brow = e.bias + col0;
@@ -196,40 +199,33 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
 #pragma unroll
       for (int j = 0; j < 32; j += 4) {
         if (j < n_valid) {
-          const float4 b = __ldg(reinterpret_cast<const float4*>(brow + j));
-          v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+          const uint4 b = __ldg(reinterpret_cast<const uint4*>(brow + j));
+          s.w[j] = b.x; s.w[j + 1] = b.y; s.w[j + 2] = b.z; s.w[j + 3] = b.w;
         }
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __ldg(brow + j);
+      for (int j = 0; j < 32; ++j) if (j < n_valid) s.w[j] = __float_as_uint(__ldg(brow + j));
     }
-    if (e.relu) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
-    }
-  } else if (e.epi == EPI_MASK) {
+  } else if (e.epi == EPI_MASK && row_ok) {
     if (e.c_dt == DT_BF16) {
-      const __nv_bfloat16* mrow = reinterpret_cast<const __nv_bfloat16*>(e.mask) + (int64_t)row * e.ldmask + col0;
+      const unsigned short* mrow = reinterpret_cast<const unsigned short*>(e.mask) + (int64_t)row * e.ldmask + col0;
       if (whole && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0)) {
 #pragma unroll
         for (int j = 0; j < 32; j += 8) {
           if (j < n_valid) {
             const uint4 q = __ldg(reinterpret_cast<const uint4*>(mrow + j));
-            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              // a bf16 is positive iff its sign bit is clear and it is not zero
-              const uint32_t lo = w[t] & 0xFFFFu, hi = w[t] >> 16;
-              if (!(lo != 0u && lo < 0x8000u)) v[j + 2 * t] = 0.f;
-              if (!(hi != 0u && hi < 0x8000u)) v[j + 2 * t + 1] = 0.f;
-            }
+            s.w[j / 2] = q.x; s.w[j / 2 + 1] = q.y; s.w[j / 2 + 2] = q.z; s.w[j / 2 + 3] = q.w;
           }
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (j < n_valid && !(__bfloat162float(mrow[j]) > 0.f)) v[j] = 0.f;
+        for (int j = 0; j < 32; j += 2) {
+          uint32_t lo = 0u, hi = 0u;
+          if (j < n_valid) lo = __ldg(mrow + j);
+          if (j + 1 < n_valid) hi = __ldg(mrow + j + 1);
+          s.w[j / 2] = lo | (hi << 16);
+        }
       }
     } else {
       const float* mrow = reinterpret_cast<const float*>(e.mask) + (int64_t)row * e.ldmask + col0;
@@ -237,18 +233,45 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
           if (j < n_valid) {
-            const float4 m = __ldg(reinterpret_cast<const float4*>(mrow + j));
-            if (!(m.x > 0.f)) v[j] = 0.f;
-            if (!(m.y > 0.f)) v[j + 1] = 0.f;
-            if (!(m.z > 0.f)) v[j + 2] = 0.f;
-            if (!(m.w > 0.f)) v[j + 3] = 0.f;
+            const uint4 m = __ldg(reinterpret_cast<const uint4*>(mrow + j));
+            s.w[j] = m.x; s.w[j + 1] = m.y; s.w[j + 2] = m.z; s.w[j + 3] = m.w;
           }
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (j < n_valid && !(__ldg(mrow + j) > 0.f)) v[j] = 0.f;
+        for (int j = 0; j < 32; ++j) if (j < n_valid) s.w[j] = __float_as_uint(__ldg(mrow + j));
       }
+    }
+  }
+}
+
+// Epilogue for up to 32 consecutive columns of one row, with the side inputs already in registers.
+// Columns are stored in groups of 8 with 16-byte accesses when the group count is whole and the
+// row segment is 16-byte aligned (every lane touches its own row, so wide accesses are what keeps
+// the number of memory wavefronts down); ragged or unaligned segments fall back to scalar stores.
+__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], const EpiSide& s, int row,
+                                               int col0, int n_total) {
+  const int n_valid = min(32, n_total - col0);
+  const bool whole = (n_valid & 7) == 0;
+  if (e.epi == EPI_BIAS_ACT) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __uint_as_float(s.w[j]);
+    if (e.relu) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+    }
+  } else if (e.epi == EPI_MASK) {
+    if (e.c_dt == DT_BF16) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        // a bf16 is positive iff its sign bit is clear and it is not zero
+        const uint32_t bits = (s.w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+        if (j < n_valid && !(bits != 0u && bits < 0x8000u)) v[j] = 0.f;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid && !(__uint_as_float(s.w[j]) > 0.f)) v[j] = 0.f;
     }
   }
   if (e.c_round == RND_TF32) {
@@ -417,16 +440,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
       const int m0 = (t % tiles_m) * BLOCK_M, n0 = (t / tiles_m) * BLOCK_N;
+      const int row = m0 + quarter * 32 + lane;
+      EpiSide side, side_next;
+      epilogue_prefetch(epi, side, row, row < M, n0, N);   // before the wait: latency off the critical path
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) { ok = false; break; }
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= N) break;              // uniform across the CTA
+        if (c + 1 < BLOCK_N / 32) epilogue_prefetch(epi, side_next, row, row < M, col0 + 32, N);
         float v[32];
         tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
-        if (row < M) epilogue_store(epi, v, row, col0, N);
+        if (row < M) epilogue_store(epi, v, side, row, col0, N);
+        side = side_next;
       }
       tc_fence_before();
       __syncwarp();
@@ -596,6 +623,9 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     const int row_in_tile = quarter * 32 + lane;
     const int row = m0 + row_in_tile;
     const int w = BLOCK_N / split;                         // columns owned by each CTA: 32, 16 or 8
+    const int own_col0 = n0 + (int)rank * w;
+    EpiSide side;                                          // side inputs of this CTA's slice, fetched ahead
+    epilogue_prefetch(epi, side, row, row < M, own_col0, min(N, own_col0 + w));
     bool ok = mbar_wait(acc_bar, 0, abort_flag, dev_status);
     tc_fence_after();
     const uint32_t slice_bytes = (uint32_t)(w * BLOCK_M * 4);
@@ -642,8 +672,7 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         for (int cs = 0; cs < 32; ++cs)
           if (cs < w) own[cs] += recv[(src * w + cs) * BLOCK_M + row_in_tile];
       }
-      const int col0 = n0 + (int)rank * w;
-      if (row < M && col0 < N) epilogue_store(epi, own, row, col0, min(N, col0 + w));
+      if (row < M && own_col0 < N) epilogue_store(epi, own, side, row, own_col0, min(N, own_col0 + w));
     }
     tc_fence_before();
   }
@@ -842,16 +871,20 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     for (int t = pair; t < n_tiles && ok; t += n_pairs) {
       const int m0 = (t % tiles_m) * PAIR_TILE_M + (int)rank * BLOCK_M;
       const int n0 = (t / tiles_m) * PAIR_TILE_N;
+      const int row = m0 + quarter * 32 + lane;
+      EpiSide side, side_next;
+      epilogue_prefetch(epi, side, row, row < M, n0, N);
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) { ok = false; break; }
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
 #pragma unroll 1
       for (int c = 0; c < PAIR_TILE_N / 32; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= N) break;
+        if (c + 1 < PAIR_TILE_N / 32) epilogue_prefetch(epi, side_next, row, row < M, col0 + 32, N);
         float v[32];
         tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * PAIR_TILE_N + c * 32), v);
-        if (row < M) epilogue_store(epi, v, row, col0, N);
+        if (row < M) epilogue_store(epi, v, side, row, col0, N);
+        side = side_next;
       }
       tc_fence_before();
       __syncwarp();
@@ -889,7 +922,7 @@ int current_device_slot() {
 bool g_init_done = false, g_init_ok = false;
 bool g_allow_splitk = true;
 bool g_allow_pairs = true;
-long g_pair_min_tiles = 96;
+long g_pair_min_tiles = 0;      // SEG_PAIR_MIN_TILES: CTA pairs exactly from this many 256 x 256 tiles on (0: cost model)
 
 // 2-D tensor map over a row-major matrix: `inner` contiguous elements per row, `outer` rows,
 // `row_stride_bytes` between rows; box = box_inner x box_outer; 128-byte swizzle (32-byte atoms
@@ -1022,23 +1055,33 @@ cudaError_t launch_pair_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, cons
   return cudaErrorNotSupported;
 }
 
-// CTA pairs pay off once there are enough 256 x 256 tiles to keep the machine busy.
-bool use_pairs(int M, int N, int K) {
-  if (!g_allow_pairs) return false;
-  if (M < 256 || N < 256 || K < 256) return false;
-  const long tiles = (long)((M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((N + PAIR_TILE_N - 1) / PAIR_TILE_N);
-  return tiles >= g_pair_min_tiles;
-}
-
-int pick_block_n(int M, int N) {
+// Kernel selection by a cost model of the main loop.  One CTA's main loop is bound by the rate at
+// which one SM's shared memory is filled (about 64 bytes per clock, measured: 24 KiB of operands per
+// k-block take 0.2 us, 32 KiB 0.27 us, 48 KiB 0.4 us); a CTA pair stages 32 KiB per CTA for the work
+// a single CTA needs 48 KiB for.  Persistent kernels run ceil(tiles / CTAs) rounds of num_k k-blocks.
+struct Choice { int kind; int block_n; double us; };      // kind 0: single CTA, 1: CTA pair
+Choice pick_kernel(int M, int N, int K, bool tf32) {
+  const int num_k = (K + (tf32 ? 32 : 64) - 1) / (tf32 ? 32 : 64);
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
-  int best = 64; long best_cost = -1;
-  for (int bn : {256, 128, 64}) {
+  Choice best{0, 64, 1e30};
+  for (int bn : {64, 128, 256}) {
     if (bn > 64 && bn / 2 >= N) continue;                  // do not use a tile twice as wide as N
     const long tiles = (long)tiles_m * ((N + bn - 1) / bn);
-    const long waves = (tiles + g_num_sms - 1) / g_num_sms;
-    const long cost = waves * (bn + 32);                   // +32: per-tile fixed overhead
-    if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+    const long rounds = (tiles + g_num_sms - 1) / g_num_sms;
+    const double per_kb = (16.0 + bn / 8.0) / 120.0;       // KiB per k-block / (KiB per us)
+    const double us = rounds * (num_k * per_kb + 0.4 + bn / 128.0);   // + per-tile epilogue not hidden
+    if (us < best.us) best = Choice{0, bn, us};
+  }
+  if (g_allow_pairs && M >= 256 && N >= 256 && K >= 256) {
+    const long tiles = (long)((M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((N + PAIR_TILE_N - 1) / PAIR_TILE_N);
+    const long pairs = g_num_sms / 2;
+    const long rounds = (tiles + pairs - 1) / pairs;
+    const double us = rounds * (num_k * (32.0 / 120.0) + 0.4 + 2.0);
+    if (g_pair_min_tiles > 0) {                            // diagnostic override: pairs from that many tiles on
+      if (tiles >= g_pair_min_tiles) best = Choice{1, PAIR_HALF_N, us};
+    } else if (us < best.us) {
+      best = Choice{1, PAIR_HALF_N, us};
+    }
   }
   return best;
 }
@@ -1091,8 +1134,9 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   if (a_pitch * (int64_t)esz >= (1ll << 40) || b_pitch * (int64_t)esz >= (1ll << 40)) return cudaErrorNotSupported;
 
   const int split = g_allow_splitk ? pick_split(g.M, g.N, g.K, tf32) : 1;
-  const bool pairs = (split == 1) && use_pairs(g.M, g.N, g.K);
-  const int block_n = split > 1 ? SPLITK_BLOCK_N : (pairs ? PAIR_HALF_N : pick_block_n(g.M, g.N));
+  const Choice choice = pick_kernel(g.M, g.N, g.K, tf32);
+  const bool pairs = (split == 1) && choice.kind == 1;
+  const int block_n = split > 1 ? SPLITK_BLOCK_N : choice.block_n;
   const uint32_t block_k = tf32 ? 32 : 64, chunk = tf32 ? 32 : 64;
   CUtensorMap ma, mb;
   bool ok;
