@@ -38,6 +38,8 @@ struct GemmDesc {
   const float* bias;        // EPI_BIAS_ACT: [N]
   const void* mask;         // EPI_MASK: [M][ldmask] of c_dt
   int64_t ldmask;
+  int off_critical_path;    // 1: the product runs beside others (a weight gradient on its branch): choose the
+                            // tiling that occupies the fewest SMs for the shortest time, not the fastest alone
 };
 
 // ---- launchers (each returns the cudaError_t of its launch) -------------------------------

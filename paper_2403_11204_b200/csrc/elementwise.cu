@@ -271,12 +271,35 @@ stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t 
     bc[0] = (float)(1.0 - pow((double)beta1, (double)step));
     bc[1] = (float)(1.0 - pow((double)beta2, (double)step));
   }
-  for (int64_t e = tid; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t r = e / cols, c = e % cols;
-    // gather_src: the input of sample r is row cls[r] of an fp32 label matrix (the fully separate variant)
-    const float raw = gather_src ? __ldg(gather_src + (int64_t)__ldg(cls_src + r) * cols + c)
-                                 : load_as_float(src, dt, r * ld_src + c);
-    store_from_float(dst, dt, r * ld_dst + c, apply_round(raw, round));
+  const int esz = dt == DT_BF16 ? 2 : 4;
+  const bool wide = gather_src == nullptr && ((cols * esz) & 15) == 0 && ((ld_src * esz) & 15) == 0 &&
+                    ((ld_dst * esz) & 15) == 0 &&
+                    ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0;
+  if (wide) {
+    // 16 bytes per access: rows are whole numbers of 16-byte groups on both sides
+    const int vec_per_row = cols * esz / 16;
+    const int64_t n_vec = (int64_t)rows * vec_per_row;
+    const char* sb = reinterpret_cast<const char*>(src);
+    char* db = reinterpret_cast<char*>(dst);
+    for (int64_t v = tid; v < n_vec; v += (int64_t)gridDim.x * blockDim.x) {
+      const int64_t r = v / vec_per_row, c = v % vec_per_row;
+      uint4 q = __ldg(reinterpret_cast<const uint4*>(sb + r * ld_src * esz) + c);
+      if (round == RND_TF32 && dt == DT_F32) {
+        q.x = __float_as_uint(round_tf32_rne(__uint_as_float(q.x)));
+        q.y = __float_as_uint(round_tf32_rne(__uint_as_float(q.y)));
+        q.z = __float_as_uint(round_tf32_rne(__uint_as_float(q.z)));
+        q.w = __float_as_uint(round_tf32_rne(__uint_as_float(q.w)));
+      }
+      reinterpret_cast<uint4*>(db + r * ld_dst * esz)[c] = q;
+    }
+  } else {
+    for (int64_t e = tid; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+      const int64_t r = e / cols, c = e % cols;
+      // gather_src: the input of sample r is row cls[r] of an fp32 label matrix (the fully separate variant)
+      const float raw = gather_src ? __ldg(gather_src + (int64_t)__ldg(cls_src + r) * cols + c)
+                                   : load_as_float(src, dt, r * ld_src + c);
+      store_from_float(dst, dt, r * ld_dst + c, apply_round(raw, round));
+    }
   }
   for (int64_t i = tid; i < rows; i += (int64_t)gridDim.x * blockDim.x) cls_dst[i] = cls_src[i];
 }
@@ -351,7 +374,8 @@ cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* s
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2,
                                 const float* gather_src, cudaStream_t s) {
-  const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
+  const int esz = dt == DT_BF16 ? 2 : 4;
+  const int grid = grid_for((int64_t)rows * cols * esz / 16, 256, 148 * 8);   // one 16-byte group per thread and pass
   launch_k(stage_inputs_kernel, dim3(grid), dim3(256), 0, s, dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
                                            beta1, beta2, gather_src);
   return cudaGetLastError();

@@ -1060,7 +1060,7 @@ cudaError_t launch_pair_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, cons
 // k-block take 0.2 us, 32 KiB 0.27 us, 48 KiB 0.4 us); a CTA pair stages 32 KiB per CTA for the work
 // a single CTA needs 48 KiB for.  Persistent kernels run ceil(tiles / CTAs) rounds of num_k k-blocks.
 struct Choice { int kind; int block_n; double us; };      // kind 0: single CTA, 1: CTA pair
-Choice pick_kernel(int M, int N, int K, bool tf32) {
+Choice pick_kernel(int M, int N, int K, bool tf32, bool throughput) {
   const int num_k = (K + (tf32 ? 32 : 64) - 1) / (tf32 ? 32 : 64);
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   Choice best{0, 64, 1e30};
@@ -1069,14 +1069,17 @@ Choice pick_kernel(int M, int N, int K, bool tf32) {
     const long tiles = (long)tiles_m * ((N + bn - 1) / bn);
     const long rounds = (tiles + g_num_sms - 1) / g_num_sms;
     const double per_kb = (16.0 + bn / 8.0) / 120.0;       // KiB per k-block / (KiB per us)
-    const double us = rounds * (num_k * per_kb + 0.4 + bn / 128.0);   // + per-tile epilogue not hidden
+    double us = rounds * (num_k * per_kb + 0.4 + bn / 128.0);   // + per-tile epilogue not hidden
+    // beside other kernels what counts is the SM time taken: tiles x (time of a tile, fixed cost included)
+    if (throughput) us = (double)tiles * (num_k * per_kb + 4.0 + bn / 128.0) / g_num_sms;
     if (us < best.us) best = Choice{0, bn, us};
   }
   if (g_allow_pairs && M >= 256 && N >= 256 && K >= 256) {
     const long tiles = (long)((M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((N + PAIR_TILE_N - 1) / PAIR_TILE_N);
     const long pairs = g_num_sms / 2;
     const long rounds = (tiles + pairs - 1) / pairs;
-    const double us = rounds * (num_k * (32.0 / 120.0) + 0.4 + 2.0);
+    double us = rounds * (num_k * (32.0 / 120.0) + 0.4 + 2.0);
+    if (throughput) us = (double)(2 * tiles) * (num_k * (32.0 / 120.0) + 9.0) / g_num_sms;   // measured: a pair's fixed cost is about 9 us
     if (g_pair_min_tiles > 0) {                            // diagnostic override: pairs from that many tiles on
       if (tiles >= g_pair_min_tiles) best = Choice{1, PAIR_HALF_N, us};
     } else if (us < best.us) {
@@ -1133,8 +1136,9 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   if ((a_pitch * esz) % 16 != 0 || (b_pitch * esz) % 16 != 0) return cudaErrorNotSupported;
   if (a_pitch * (int64_t)esz >= (1ll << 40) || b_pitch * (int64_t)esz >= (1ll << 40)) return cudaErrorNotSupported;
 
-  const int split = g_allow_splitk ? pick_split(g.M, g.N, g.K, tf32) : 1;
-  const Choice choice = pick_kernel(g.M, g.N, g.K, tf32);
+  const bool throughput = g.off_critical_path != 0;
+  const int split = (g_allow_splitk && !throughput) ? pick_split(g.M, g.N, g.K, tf32) : 1;
+  const Choice choice = pick_kernel(g.M, g.N, g.K, tf32, throughput);
   const bool pairs = (split == 1) && choice.kind == 1;
   const int block_n = split > 1 ? SPLITK_BLOCK_N : choice.block_n;
   const uint32_t block_k = tf32 ? 32 : 64, chunk = tf32 ? 32 : 64;

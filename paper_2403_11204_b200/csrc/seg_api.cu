@@ -529,6 +529,7 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
     w.B = a_prev; w.b_sk = ld_prev; w.b_sn = 1; w.b_dt = h->act_dt;
     w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
     w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
+    w.off_critical_path = l > 0;  // the upper layers' weight gradients run beside the dgrad chain and each other
     if ((st = run_gemm(h, w, K_WGRAD, ls)) != SEG_OK) return st;
     // update of W_l and b_l (adjacent in the flat range) once dgrad(l) no longer reads the old W_l
     if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
