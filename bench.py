@@ -353,23 +353,36 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
                                "peak_source": f"{peaks['source']}: copy bandwidth",
                                "timing": "CUDA events around every launch of this kind, same steps re-run after the timed region",
                                "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
-        # end to end: pinned host batches in, loss out, every step
+        # end to end through the host-buffer entry points: every step reads its batch from pinned host memory
+        # (host -> device inside the step) and writes its loss to pinned host memory (device -> host).
+        # Timed twice: seg_train_step_host_async (steps enqueued back to back, one synchronisation at the end:
+        # how a training loop calls it) and seg_train_step_host (waits for every loss).
         e_steps = max(3, min(steps, 50))
-        for s in range(3):
-            sl = r.batch_slice(s)
-            for k, seg in enumerate(r.segs):
-                seg.train_step_host(r.host_x[k][sl], r.host_cls[sl])
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for s in range(e_steps):
-            sl = r.batch_slice(s + 3)
-            for k, seg in enumerate(r.segs):
-                seg.train_step_host(r.host_x[k][sl], r.host_cls[sl])
-        torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
         h2d = sum(w.batch * (spec.widths[0] * (2 if w.precision == "bf16" else 4) + 4) for spec in w.segments)
-        out["e2e"] = {"value": e_steps * w.batch / dt, "unit": "samples/s", "h2d_bytes_per_step": h2d,
-                      "d2h_bytes_per_step": 4 * len(w.segments), "steps": e_steps}
+        loss_pin = torch.zeros(e_steps + 3, len(r.segs), dtype=torch.float32).pin_memory()
+
+        def e2e_loop(sync_every_step):
+            for s in range(3 + e_steps):
+                if s == 3:
+                    torch.cuda.synchronize()
+                    t0 = time.perf_counter()
+                sl = r.batch_slice(s)
+                for k, seg in enumerate(r.segs):
+                    if sync_every_step:
+                        seg.train_step_host(r.host_x[k][sl], r.host_cls[sl])
+                    else:
+                        seg.train_step_host_async(r.host_x[k][sl], r.host_cls[sl], loss_pin[s, k:k + 1])
+            torch.cuda.synchronize()
+            return time.perf_counter() - t0
+
+        dt_sync = e2e_loop(True)
+        dt_async = e2e_loop(False)
+        assert bool(torch.isfinite(loss_pin[3:]).all()) and float(loss_pin[3:].abs().sum()) > 0.0
+        out["e2e"] = {"value": e_steps * w.batch / dt_async, "unit": "samples/s", "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": 4 * len(w.segments), "steps": e_steps,
+                      "call": "seg_train_step_host_async per segment and step, one synchronisation after the last step",
+                      "waiting_for_every_loss": {"value": e_steps * w.batch / dt_sync, "unit": "samples/s",
+                                                 "call": "seg_train_step_host"}}
     if full and not w.concurrent:
         # the whole procedure of Section 2, one epoch per segment: train segment k over the resident set in
         # stored order (last partial batch included), store its response, hand it to segment k+1

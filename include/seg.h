@@ -147,12 +147,22 @@ SEG_API seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* c
 SEG_API seg_status seg_train_step_label_input(seg_handle* h, const float* sil_in, const int32_t* cls,
                                               int32_t batch, float* loss_out);
 
-/* The same step for callers whose batch lives in HOST memory: copies x_host and cls_host
- * (host pointers; page-locked memory gives full copy speed) to device buffers the handle
- * owns (allocated at the first such call), runs seg_train_step, copies the loss back to
- * *loss_host (host float, may be NULL) and synchronises the stream before returning.     */
+/* The same step for callers whose batch lives in HOST memory (x_host, cls_host: host pointers).
+ * Page-locked (pinned, mapped) buffers are read by the step's staging kernel directly over the bus;
+ * pageable ones are first copied to device buffers the handle owns (allocated at the first such
+ * call).  The loss is written by the kernel into a page-locked float of the handle and returned in
+ * *loss_host (host float, may be NULL); the call synchronises the stream before returning.       */
 SEG_API seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t* cls_host,
                                        int32_t batch, float* loss_host);
+
+/* The host-buffer step without the wait, for training loops that keep the GPU fed: x_host, cls_host
+ * and loss_host (may be NULL) must all be page-locked, mapped host memory (SEG_ERR_INVALID_ARG
+ * otherwise).  The call enqueues the step and returns; the staging kernel reads the batch from host
+ * memory when the step runs and the loss kernel writes *loss_host when it is done, so the caller
+ * leaves the batch unchanged, and does not read the loss, until the stream has passed that step
+ * (seg_poll_status, or a synchronisation of the handle's stream).                                 */
+SEG_API seg_status seg_train_step_host_async(seg_handle* h, const void* x_host, const int32_t* cls_host,
+                                             int32_t batch, float* loss_host);
 
 /* Forward pass only (the response handed to the next segment, Section 2):
  *   y [batch][widths[n_layers]]: float for FP32/TF32 and for the logits of a final

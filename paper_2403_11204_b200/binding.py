@@ -39,6 +39,7 @@ EXPORTS = {
     "seg_train_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
     "seg_train_step_label_input": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_train_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_float)]),
+    "seg_train_step_host_async": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_forward": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_recovery_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "seg_train_epochs": (c_int32, [c_void_p, c_void_p, c_void_p, ctypes.c_int64, c_int32, c_int32, c_void_p]),
@@ -237,6 +238,18 @@ class Segment:
                     "seg_train_step_host")
         self.last_batch = batch
         return loss.value
+
+    def train_step_host_async(self, x_host, cls_host, loss_host=None):
+        """seg_train_step_host_async: pinned CPU tensors in, nothing waited for.  loss_host: a pinned
+        float32 CPU tensor (one element) the step's loss is written to when the step has run."""
+        batch = x_host.shape[0]
+        assert not x_host.is_cuda and x_host.is_contiguous() and x_host.dtype == self.act_dtype
+        assert not cls_host.is_cuda and cls_host.dtype == self._torch.int32
+        lp = None if loss_host is None else c_void_p(loss_host.data_ptr())
+        self._check(self.lib.seg_train_step_host_async(self.h, c_void_p(x_host.data_ptr()),
+                                                       c_void_p(cls_host.data_ptr()), batch, lp),
+                    "seg_train_step_host_async")
+        self.last_batch = batch
 
     def forward(self, x, y=None):
         batch = x.shape[0]

@@ -100,7 +100,8 @@ struct seg_handle {
   int* dev_status = nullptr;
   void* host_x = nullptr;          // device staging of seg_train_step_host
   int32_t* host_cls = nullptr;
-  float* host_loss = nullptr;
+  float* host_loss = nullptr;      // page-locked host float the loss kernel writes (seg_train_step_host)
+  float* host_loss_dev = nullptr;  // its device-side address
   int last_batch = 0;
   uint64_t step = 0;
   uint64_t mem_current = 0, mem_peak = 0, launches = 0;
@@ -415,6 +416,7 @@ seg_status seg_destroy(seg_handle* h) {
   for (cudaEvent_t e : h->ev_done) if (e) cudaEventDestroy(e);
   for (cudaStream_t ls : h->lstream) if (ls) cudaStreamDestroy(ls);
   for (void* p : h->allocations) cudaFree(p);
+  if (h->host_loss) cudaFreeHost(h->host_loss);
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->ev_start) cudaEventDestroy(h->ev_start);
   if (h->ev_stop) cudaEventDestroy(h->ev_stop);
@@ -747,26 +749,67 @@ seg_status seg_forward_dataset(seg_handle* h, const void* x, int64_t n, int32_t 
   return SEG_OK;
 }
 
+// Device-side address of a page-locked, mapped host buffer (what cudaHostAlloc, cudaHostRegister and
+// torch's pinned tensors give); nullptr for pageable memory.
+static const void* mapped_device_pointer(const void* host) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (a.type != cudaMemoryTypeHost || a.devicePointer == nullptr) return nullptr;
+  return a.devicePointer;
+}
+
 seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t* cls_host, int32_t batch,
                                float* loss_host) {
   if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   seg_status st;
   const size_t row_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
-  if (!h->host_x) {
+  // Page-locked batches are read by the staging kernel straight from host memory (the transfer happens
+  // inside that kernel, no separate copy is enqueued); pageable ones go through a device buffer.
+  const void* x_dev = mapped_device_pointer(x_host);
+  const int32_t* cls_dev = reinterpret_cast<const int32_t*>(mapped_device_pointer(cls_host));
+  if ((!x_dev || !cls_dev) && !h->host_x) {
     char* p = nullptr;
     if ((st = dev_alloc(h, &p, (size_t)h->max_batch * row_bytes, false)) != SEG_OK) return st;
     h->host_x = p;
     if ((st = dev_alloc(h, &h->host_cls, h->max_batch, false)) != SEG_OK) return st;
-    if ((st = dev_alloc(h, &h->host_loss, 1, true)) != SEG_OK) return st;
   }
-  SEG_TRY(h, cudaMemcpyAsync(h->host_x, x_host, batch * row_bytes, cudaMemcpyHostToDevice, h->stream), "input copy");
-  SEG_TRY(h, cudaMemcpyAsync(h->host_cls, cls_host, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, h->stream), "class copy");
-  if ((st = seg_train_step(h, h->host_x, h->host_cls, batch, h->host_loss, nullptr)) != SEG_OK) return st;
-  if (loss_host)
-    SEG_TRY(h, cudaMemcpyAsync(loss_host, h->host_loss, sizeof(float), cudaMemcpyDeviceToHost, h->stream), "loss copy");
+  if (!h->host_loss) {
+    // the loss lands in page-locked host memory the kernel writes directly: no copy back, one synchronisation
+    void* p = nullptr;
+    SEG_TRY(h, cudaHostAlloc(&p, sizeof(float), cudaHostAllocMapped), "page-locked loss slot");
+    h->host_loss = reinterpret_cast<float*>(p);
+    void* d = nullptr;
+    SEG_TRY(h, cudaHostGetDevicePointer(&d, p, 0), "page-locked loss slot");
+    h->host_loss_dev = reinterpret_cast<float*>(d);
+  }
+  if (!x_dev) {
+    SEG_TRY(h, cudaMemcpyAsync(h->host_x, x_host, batch * row_bytes, cudaMemcpyHostToDevice, h->stream), "input copy");
+    x_dev = h->host_x;
+  }
+  if (!cls_dev) {
+    SEG_TRY(h, cudaMemcpyAsync(h->host_cls, cls_host, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, h->stream), "class copy");
+    cls_dev = h->host_cls;
+  }
+  if ((st = seg_train_step(h, x_dev, cls_dev, batch, h->host_loss_dev, nullptr)) != SEG_OK) return st;
   SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
+  if (loss_host) *loss_host = *reinterpret_cast<volatile float*>(h->host_loss);
   return SEG_OK;
+}
+
+seg_status seg_train_step_host_async(seg_handle* h, const void* x_host, const int32_t* cls_host, int32_t batch,
+                                     float* loss_host) {
+  if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
+  if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
+  const void* x_dev = mapped_device_pointer(x_host);
+  const int32_t* cls_dev = reinterpret_cast<const int32_t*>(mapped_device_pointer(cls_host));
+  float* loss_dev = nullptr;
+  if (loss_host) {
+    loss_dev = reinterpret_cast<float*>(const_cast<void*>(mapped_device_pointer(loss_host)));
+    if (!loss_dev) return SEG_ERR_INVALID_ARG;
+  }
+  if (!x_dev || !cls_dev) return SEG_ERR_INVALID_ARG;      // pageable memory cannot be read while the host runs on
+  return seg_train_step(h, x_dev, cls_dev, batch, loss_dev, nullptr);
 }
 
 seg_status seg_get_labels(seg_handle* h, float* dst) {

@@ -126,16 +126,49 @@ def test_forward_only_and_set_params_route():
     gpu.close()
 
 
-def test_host_buffer_step_matches_device_step():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_step_matches_device_step(pinned):
+    """Page-locked batches are read by the staging kernel straight from host memory, pageable ones go
+    through a device copy; both must give the oracle's step, two steps in a row (second batch differs)."""
     import torch
     w = wl.WORKLOADS["tiny"]
     a, ora = make_pair([784, 128, 128, 64], 47, False, "fp32", "sgd", 0.01, 64)
-    x, cls = batch_arrays(w, 64, 784)
-    loss = a.train_step_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(cls.astype(np.int32)).pin_memory())
-    ref = ora.train_step(x, cls)
-    assert abs(loss - ref) / abs(ref) < 1e-4
+    x, cls = batch_arrays(w, 128, 784)
+    for lo in (0, 64):
+        xb, cb = x[lo:lo + 64].copy(), cls[lo:lo + 64].astype(np.int32)
+        xt, ct = torch.from_numpy(xb), torch.from_numpy(cb)
+        if pinned:
+            xt, ct = xt.pin_memory(), ct.pin_memory()
+        loss = a.train_step_host(xt, ct)
+        ref = ora.train_step(xb, cls[lo:lo + 64])
+        assert abs(loss - ref) / abs(ref) < 1e-4
     W, _ = a.params(0)
     assert rel_err(W.cpu().numpy(), ora.W[0]) < 1e-4
+    a.close()
+
+
+def test_host_buffer_step_without_wait():
+    """seg_train_step_host_async: three steps enqueued back to back from pinned batches, losses read after
+    one synchronisation; pageable buffers are refused."""
+    import torch
+    from paper_2403_11204_b200.binding import SegError
+    w = wl.WORKLOADS["tiny"]
+    a, ora = make_pair([784, 128, 128, 64], 47, False, "fp32", "sgd", 0.01, 64)
+    x, cls = batch_arrays(w, 192, 784)
+    xs = torch.from_numpy(x).pin_memory()
+    cs = torch.from_numpy(cls.astype(np.int32)).pin_memory()
+    losses = torch.zeros(3, dtype=torch.float32).pin_memory()
+    for i in range(3):
+        a.train_step_host_async(xs[64 * i:64 * (i + 1)], cs[64 * i:64 * (i + 1)], losses[i:i + 1])
+    a.poll()
+    for i in range(3):
+        ref = ora.train_step(x[64 * i:64 * (i + 1)], cls[64 * i:64 * (i + 1)])
+        assert abs(float(losses[i]) - ref) / abs(ref) < 1e-4
+    W, _ = a.params(0)
+    assert rel_err(W.cpu().numpy(), ora.W[0]) < 1e-4
+    with pytest.raises(SegError) as e:
+        a.train_step_host_async(torch.from_numpy(x[:64].copy()), cs[:64])
+    assert e.value.status == 1
     a.close()
 
 
