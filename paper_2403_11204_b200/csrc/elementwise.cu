@@ -156,40 +156,43 @@ __device__ __forceinline__ void opt_step(float& p, float g, float& m, float& v, 
 
 // The update of one layer in one launch.  Parameters, gradients and optimizer state share one flat
 // layout [W | b]:
-//   blocks [0, bias_blocks): each forms the bias gradient of 32 columns, db[n] = sum_b dZ[b][n]
-//     (8 row lanes per column, then the lanes in index order: one fixed order, bit-reproducible),
+//   blocks [0, bias_blocks): each forms the bias gradient of 8 or 32 columns, db[n] = sum_b dZ[b][n]
+//     (32 or 8 row lanes per column, then the lanes in index order: one fixed order, bit-reproducible),
 //     stores it and applies the optimizer to those bias elements;
 //   the other blocks stream over the weight range, whose gradient the weight-gradient product wrote.
 // Both parts refresh the reduced-precision operand copy.
 template <int OPT, int OPDT>
 __global__ void __launch_bounds__(256)
-update_kernel(UpdateArgs u, int bias_blocks) {
+update_kernel(UpdateArgs u, int bias_blocks, int bias_cols) {
   pdl_wait();
   pdl_trigger();
   float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
   if constexpr (OPT == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(u.bc); inv_bc2 = 1.0f / __ldg(u.bc + 1); }
   if ((int)blockIdx.x < bias_blocks) {
-    __shared__ float part[8][33];
-    const int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
-    const int col = blockIdx.x * 32 + lane;
+    // small batches: 8 columns x 32 row lanes per block, so that the walk over the batch is only batch / 32
+    // loads deep and these blocks finish inside the streaming part even when the layer is small;
+    // large batches: 32 columns x 8 row lanes (whole 64- or 128-byte row segments per warp)
+    __shared__ float part[32][33];
+    const int cols = bias_cols, lanes = 256 / bias_cols;
+    const int c = threadIdx.x % cols, rl = threadIdx.x / cols;
+    const int col = blockIdx.x * cols + c;
     float acc = 0.f;
     if (col < u.n_bias) {
       if (u.dz_dt == DT_BF16) {
         const __nv_bfloat16* dz = reinterpret_cast<const __nv_bfloat16*>(u.dz);
 #pragma unroll 8
-        for (int b = rl; b < u.batch; b += 8) acc += __bfloat162float(dz[(int64_t)b * u.ld_dz + col]);
+        for (int b = rl; b < u.batch; b += lanes) acc += __bfloat162float(dz[(int64_t)b * u.ld_dz + col]);
       } else {
         const float* dz = reinterpret_cast<const float*>(u.dz);
 #pragma unroll 8
-        for (int b = rl; b < u.batch; b += 8) acc += dz[(int64_t)b * u.ld_dz + col];
+        for (int b = rl; b < u.batch; b += lanes) acc += dz[(int64_t)b * u.ld_dz + col];
       }
     }
-    part[rl][lane] = acc;
+    part[rl][c] = acc;
     __syncthreads();
     if (rl == 0 && col < u.n_bias) {
       float g = 0.f;
-#pragma unroll
-      for (int r = 0; r < 8; ++r) g += part[r][lane];
+      for (int r = 0; r < lanes; ++r) g += part[r][c];
       const int64_t i = u.bias_off + col;
       u.g_bias[col] = g;
       float p = u.p[i], m = 0.f, v = 0.f;
@@ -353,13 +356,14 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
 
 cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
   if (u.n & 3) return cudaErrorInvalidValue;
-  const int bias_blocks = (u.dz != nullptr && u.n_bias > 0) ? (u.n_bias + 31) / 32 : 0;
+  const int bias_cols = u.batch <= 1024 ? 8 : 32;
+  const int bias_blocks = (u.dz != nullptr && u.n_bias > 0) ? (u.n_bias + bias_cols - 1) / bias_cols : 0;
   if (u.n == 0 && bias_blocks == 0) return cudaSuccess;
   const int grid = bias_blocks + (u.n > 0 ? grid_for(u.n >> 2, 256, 148 * 8) : 0);
   const bool bf = (u.p_op != nullptr && u.op_dt == DT_BF16);
 #define SEGK_UPD(OPT)                                                      \
-  if (bf) launch_k(update_kernel<OPT, DT_BF16>, dim3(grid), dim3(256), 0, s, u, bias_blocks);             \
-  else launch_k(update_kernel<OPT, DT_F32>, dim3(grid), dim3(256), 0, s, u, bias_blocks)
+  if (bf) launch_k(update_kernel<OPT, DT_BF16>, dim3(grid), dim3(256), 0, s, u, bias_blocks, bias_cols);             \
+  else launch_k(update_kernel<OPT, DT_F32>, dim3(grid), dim3(256), 0, s, u, bias_blocks, bias_cols)
   switch (u.optimizer) {
     case SEG_SGD: SEGK_UPD(SEG_SGD); break;
     case SEG_SGD_MOMENTUM: SEGK_UPD(SEG_SGD_MOMENTUM); break;
