@@ -40,10 +40,18 @@ struct GemmDesc {
   int64_t ldmask;
   int off_critical_path;    // 1: the product runs beside others (a weight gradient on its branch): choose the
                             // tiling that occupies the fewest SMs for the shortest time, not the fastest alone
+  // FFMA path only: workspace for splitting K over several CTAs of one tile (may be null: no split).
+  // simt_scratch holds simt_slots partial tiles of 64 x 64 floats, simt_counters one arrival counter
+  // per slot (zero between launches).  Products that may run at the same time need separate workspaces.
+  float* simt_scratch;
+  unsigned int* simt_counters;
+  int simt_slots;
 };
+constexpr int kSimtTileFloats = 64 * 64;
 
 // ---- launchers (each returns the cudaError_t of its launch) -------------------------------
 cudaError_t launch_gemm_simt(const GemmDesc& g, cudaStream_t s);
+int gemm_simt_slots(int M, int N, int K);   // workspace slots (partial 64 x 64 tiles) a split of this product would use
 // Tensor-core path.  Returns cudaErrorNotSupported when the shape/stride does not fit its TMA rules.
 cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s);
 bool gemm_tc_init();   // resolves the driver entry point needed for tensor maps

@@ -72,6 +72,11 @@ struct seg_handle {
   float* loss_slot = nullptr;
   unsigned long long* step_dev = nullptr;
   float* bc_dev = nullptr;
+  // FFMA path: split-K workspaces.  Index 0 serves the main branch (its products run one after another),
+  // index l >= 1 the weight gradient of layer l, which runs on its own branch.
+  std::vector<float*> simt_scratch;
+  std::vector<unsigned int*> simt_counters;
+  std::vector<int> simt_slots;
   std::vector<cudaStream_t> lstream;  // lstream[l], l >= 1: the branch of layer l (weight gradient, then update)
   std::vector<cudaEvent_t> ev_dz;     // ev_dz[l]: dZ_l is complete (main branch)
   std::vector<cudaEvent_t> ev_done;   // ev_done[l], l >= 1: layer l's branch is complete
@@ -168,10 +173,15 @@ struct Launch {
   }
 };
 
-seg_status run_gemm(seg_handle* h, const GemmDesc& g_in, int kind, cudaStream_t stream, bool* used_tc = nullptr) {
+seg_status run_gemm(seg_handle* h, const GemmDesc& g_in, int kind, cudaStream_t stream, bool* used_tc = nullptr,
+                    int workspace = 0) {
   Launch l(h, kind, stream);
   if (used_tc) *used_tc = false;
   GemmDesc g = g_in;
+  if (workspace < (int)h->simt_scratch.size() && h->simt_scratch[workspace]) {
+    g.simt_scratch = h->simt_scratch[workspace]; g.simt_counters = h->simt_counters[workspace];
+    g.simt_slots = h->simt_slots[workspace];
+  }
   if (h->use_tc) {
     cudaError_t e = launch_gemm_tc(g, h->dev_status, stream);
     if (e == cudaSuccess) { if (used_tc) *used_tc = true; return SEG_OK; }
@@ -381,6 +391,26 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
     env = getenv("SEG_NO_FORK");
     if (env && env[0] == '1') h->fork_enabled = false;
   }
+  if (!h->use_tc) {
+    // split-K workspaces of the FFMA path, sized for the products each one serves at max_batch
+    h->simt_scratch.assign(h->n_layers, nullptr);
+    h->simt_counters.assign(h->n_layers, nullptr);
+    h->simt_slots.assign(h->n_layers, 0);
+    const int B = h->max_batch;
+    for (int l = 0; l < h->n_layers; ++l) {
+      const int in = h->widths[l], out = h->widths[l + 1];
+      const int wg = gemm_simt_slots(out, in, B);
+      if (l > 0) h->simt_slots[l] = wg;
+      else h->simt_slots[0] = std::max(h->simt_slots[0], wg);
+      h->simt_slots[0] = std::max(h->simt_slots[0], gemm_simt_slots(B, out, in));            // forward
+      if (l > 0) h->simt_slots[0] = std::max(h->simt_slots[0], gemm_simt_slots(B, in, out)); // dgrad
+    }
+    for (int l = 0; l < h->n_layers; ++l) {
+      if (h->simt_slots[l] == 0) continue;
+      if ((st = dev_alloc(h, &h->simt_scratch[l], (size_t)h->simt_slots[l] * kSimtTileFloats, false)) != SEG_OK) return bail(st);
+      if ((st = dev_alloc(h, &h->simt_counters[l], h->simt_slots[l], true)) != SEG_OK) return bail(st);
+    }
+  }
   if (!h->is_final &&
       (st = dev_alloc(h, &h->sil, (size_t)h->n_classes * h->widths[h->n_layers], true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->loss_partials, loss_max_partials(), true)) != SEG_OK) return bail(st);
@@ -532,7 +562,7 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
     w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
     w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
     w.off_critical_path = l > 0;  // the upper layers' weight gradients run beside the dgrad chain and each other
-    if ((st = run_gemm(h, w, K_WGRAD, ls)) != SEG_OK) return st;
+    if ((st = run_gemm(h, w, K_WGRAD, ls, nullptr, l)) != SEG_OK) return st;
     // update of W_l and b_l (adjacent in the flat range) once dgrad(l) no longer reads the old W_l
     if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
     const int64_t lo = Ly.w_off;
