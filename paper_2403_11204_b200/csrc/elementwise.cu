@@ -356,7 +356,7 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
 
 cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
   if (u.n & 3) return cudaErrorInvalidValue;
-  const int bias_cols = u.batch <= 1024 ? 8 : 32;
+  const int bias_cols = (u.batch <= 1024 || u.n_bias <= 256) ? 8 : 32;   // narrow layers: few blocks either way, keep the walk short
   const int bias_blocks = (u.dz != nullptr && u.n_bias > 0) ? (u.n_bias + bias_cols - 1) / bias_cols : 0;
   if (u.n == 0 && bias_blocks == 0) return cudaSuccess;
   const int grid = bias_blocks + (u.n > 0 ? grid_for(u.n >> 2, 256, 148 * 8) : 0);
