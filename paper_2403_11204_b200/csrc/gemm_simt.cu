@@ -14,7 +14,7 @@
 namespace segk {
 namespace {
 
-constexpr int BM = 64, BN = 64, BK = 16, PAD = 4;
+constexpr int BM = 64, BN = 64, BK = 32, PAD = 4;
 
 template <typename T>
 __device__ __forceinline__ float to_f(T v);
@@ -38,26 +38,37 @@ gemm_simt_kernel(GemmDesc g, int k_per_split) {
   const bool a_kfast = (g.a_sk == 1), b_nfast = (g.b_sn == 1);
   float acc[4][4] = {};
   const int k_begin = blockIdx.z * k_per_split, k_end = min(g.K, k_begin + k_per_split);
-  for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+  constexpr int LD = BM * BK / 256;          // elements of each operand tile a thread fetches per k-step
+  float ra[LD], rb[LD];
+  // fetch of one k-step into registers; the next step's fetch is issued before this step's arithmetic
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < LD; ++i) {
       const int idx = threadIdx.x + 256 * i;
       const int k = a_kfast ? (idx & (BK - 1)) : (idx / BM);
       const int m = a_kfast ? (idx / BK) : (idx & (BM - 1));
-      float v = 0.f;
-      if (m0 + m < g.M && k0 + k < k_end) v = to_f<TIn>(A[(int64_t)(m0 + m) * g.a_sm + (int64_t)(k0 + k) * g.a_sk]);
-      As[k][m] = v;
+      ra[i] = 0.f;
+      if (m0 + m < g.M && k0 + k < k_end) ra[i] = to_f<TIn>(A[(int64_t)(m0 + m) * g.a_sm + (int64_t)(k0 + k) * g.a_sk]);
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < LD; ++i) {
       const int idx = threadIdx.x + 256 * i;
       const int n = b_nfast ? (idx & (BN - 1)) : (idx / BK);
       const int k = b_nfast ? (idx / BN) : (idx & (BK - 1));
-      float v = 0.f;
-      if (n0 + n < g.N && k0 + k < k_end) v = to_f<TIn>(B[(int64_t)(k0 + k) * g.b_sk + (int64_t)(n0 + n) * g.b_sn]);
-      Bs[k][n] = v;
+      rb[i] = 0.f;
+      if (n0 + n < g.N && k0 + k < k_end) rb[i] = to_f<TIn>(B[(int64_t)(k0 + k) * g.b_sk + (int64_t)(n0 + n) * g.b_sn]);
+    }
+  };
+  if (k_begin < k_end) fetch(k_begin);
+  for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+#pragma unroll
+    for (int i = 0; i < LD; ++i) {
+      const int idx = threadIdx.x + 256 * i;
+      As[a_kfast ? (idx & (BK - 1)) : (idx / BM)][a_kfast ? (idx / BK) : (idx & (BM - 1))] = ra[i];
+      Bs[b_nfast ? (idx / BN) : (idx & (BK - 1))][b_nfast ? (idx & (BN - 1)) : (idx / BK)] = rb[i];
     }
     __syncthreads();
+    if (k0 + BK < k_end) fetch(k0 + BK);
 #pragma unroll
     for (int k = 0; k < BK; ++k) {
       const float4 a = *reinterpret_cast<const float4*>(&As[k][ty * 4]);

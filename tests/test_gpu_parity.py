@@ -172,6 +172,35 @@ def test_host_buffer_step_without_wait():
     a.close()
 
 
+@pytest.mark.parametrize("widths,final,precision,batch", [([784, 80, 60], False, "fp32", 1410),
+                                                          ([60, 60, 60, 47], True, "fp32", 1410),
+                                                          ([784, 1024, 512], False, "tf32", 256),
+                                                          ([512, 256, 47], True, "bf16", 200)])
+def test_step_is_bit_reproducible(widths, final, precision, batch):
+    """Every reduction of the step runs in a fixed order (loss partials, bias gradient, the K split of the
+    FFMA and tensor-core products): two handles given the same batches end with identical bits."""
+    import torch
+    w = wl.WORKLOADS["paper_net"]
+    x, cls = batch_arrays(w, batch, widths[0], precision=precision)
+    results = []
+    for _ in range(2):
+        gpu, _ = make_pair(widths, 47, final, precision, "momentum", 0.01, batch)
+        xt, ct = to_device(x, cls, precision)
+        loss = torch.zeros(3, device="cuda")
+        for i in range(3):
+            gpu.train_step(xt, ct, loss[i:i + 1])
+        gpu.poll()
+        tensors = [loss.cpu().numpy()]
+        for l in range(len(widths) - 1):
+            W, b = gpu.params(l)
+            dW, db = gpu.grads(l)
+            tensors += [W.cpu().numpy(), b.cpu().numpy(), dW.cpu().numpy(), db.cpu().numpy()]
+        results.append(tensors)
+        gpu.close()
+    for a, b in zip(*results):
+        assert bits_equal(a, b)
+
+
 def test_argument_errors_and_state():
     import torch
     from paper_2403_11204_b200.binding import SegError, Segment
