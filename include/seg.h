@@ -157,10 +157,11 @@ SEG_API seg_status seg_train_step_host(seg_handle* h, const void* x_host, const 
 
 /* The host-buffer step without the wait, for training loops that keep the GPU fed: x_host, cls_host
  * and loss_host (may be NULL) must all be page-locked, mapped host memory (SEG_ERR_INVALID_ARG
- * otherwise).  The call enqueues the step and returns; the staging kernel reads the batch from host
- * memory when the step runs and the loss kernel writes *loss_host when it is done, so the caller
- * leaves the batch unchanged, and does not read the loss, until the stream has passed that step
- * (seg_poll_status, or a synchronisation of the handle's stream).                                 */
+ * otherwise).  The call enqueues a copy of the batch on a copy stream of the handle (into one of two
+ * device buffers, allocated at the first such call, so that the transfer overlaps the steps enqueued
+ * before it), enqueues the step behind that copy and returns; the loss kernel writes *loss_host when
+ * the step is done.  The caller leaves the batch unchanged, and does not read the loss, until the
+ * stream has passed that step (seg_poll_status, or a synchronisation of the handle's stream).      */
 SEG_API seg_status seg_train_step_host_async(seg_handle* h, const void* x_host, const int32_t* cls_host,
                                              int32_t batch, float* loss_host);
 

@@ -38,8 +38,8 @@ struct GemmDesc {
   const float* bias;        // EPI_BIAS_ACT: [N]
   const void* mask;         // EPI_MASK: [M][ldmask] of c_dt
   int64_t ldmask;
-  int off_critical_path;    // 1: the product runs beside others (a weight gradient on its branch): choose the
-                            // tiling that occupies the fewest SMs for the shortest time, not the fastest alone
+  int off_critical_path;    // 1: the product runs beside others (a weight gradient on its branch): the tiling is
+                            // chosen for latency plus the SM time it takes away from them, not for latency alone
   // FFMA path only: workspace for splitting K over several CTAs of one tile (may be null: no split).
   // simt_scratch holds simt_slots partial tiles of 64 x 64 floats, simt_counters one arrival counter
   // per slot (zero between launches).  Products that may run at the same time need separate workspaces.

@@ -1070,8 +1070,12 @@ Choice pick_kernel(int M, int N, int K, bool tf32, bool throughput) {
     const long rounds = (tiles + g_num_sms - 1) / g_num_sms;
     const double per_kb = (16.0 + bn / 8.0) / 120.0;       // KiB per k-block / (KiB per us)
     double us = rounds * (num_k * per_kb + 0.4 + bn / 128.0);   // + per-tile epilogue not hidden
-    // beside other kernels what counts is the SM time taken: tiles x (time of a tile, fixed cost included)
-    if (throughput) us = (double)tiles * (num_k * per_kb + 4.0 + bn / 128.0) / g_num_sms;
+    // beside other kernels the SM time taken counts as well: latency + tiles x time of a tile / SMs, with the
+    // measured fixed cost of a tile (wider tiles drain more columns and allocate more tensor memory)
+    if (throughput) {
+      const double t = num_k * per_kb + 3.5 + bn / 48.0;
+      us = rounds * t + (double)tiles * t / g_num_sms;
+    }
     if (us < best.us) best = Choice{0, bn, us};
   }
   if (g_allow_pairs && M >= 256 && N >= 256 && K >= 256) {
@@ -1079,7 +1083,10 @@ Choice pick_kernel(int M, int N, int K, bool tf32, bool throughput) {
     const long pairs = g_num_sms / 2;
     const long rounds = (tiles + pairs - 1) / pairs;
     double us = rounds * (num_k * (32.0 / 120.0) + 0.4 + 2.0);
-    if (throughput) us = (double)(2 * tiles) * (num_k * (32.0 / 120.0) + 9.0) / g_num_sms;   // measured: a pair's fixed cost is about 9 us
+    if (throughput) {
+      const double t = num_k * (32.0 / 120.0) + 9.0;          // measured: a pair's fixed cost is about 9 us
+      us = rounds * t + (double)(2 * tiles) * t / g_num_sms;
+    }
     if (g_pair_min_tiles > 0) {                            // diagnostic override: pairs from that many tiles on
       if (tiles >= g_pair_min_tiles) best = Choice{1, PAIR_HALF_N, us};
     } else if (us < best.us) {

@@ -107,6 +107,13 @@ struct seg_handle {
   int32_t* host_cls = nullptr;
   float* host_loss = nullptr;      // page-locked host float the loss kernel writes (seg_train_step_host)
   float* host_loss_dev = nullptr;  // its device-side address
+  // seg_train_step_host_async: copy stream, two device buffers for the batch in flight and the next one
+  cudaStream_t copy_stream = nullptr;
+  void* async_x[2] = {nullptr, nullptr};
+  int32_t* async_cls[2] = {nullptr, nullptr};
+  cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
+  bool async_used[2] = {false, false};
+  int async_next = 0;
   int last_batch = 0;
   uint64_t step = 0;
   uint64_t mem_current = 0, mem_peak = 0, launches = 0;
@@ -436,6 +443,7 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
 
 seg_status seg_destroy(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
   cudaStreamSynchronize(h->stream);
   for (cudaStream_t ls : h->lstream) if (ls) cudaStreamSynchronize(ls);
   for (auto& kv : h->graphs) {
@@ -447,6 +455,11 @@ seg_status seg_destroy(seg_handle* h) {
   for (cudaStream_t ls : h->lstream) if (ls) cudaStreamDestroy(ls);
   for (void* p : h->allocations) cudaFree(p);
   if (h->host_loss) cudaFreeHost(h->host_loss);
+  for (int i = 0; i < 2; ++i) {
+    if (h->ev_copied[i]) cudaEventDestroy(h->ev_copied[i]);
+    if (h->ev_consumed[i]) cudaEventDestroy(h->ev_consumed[i]);
+  }
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->ev_start) cudaEventDestroy(h->ev_start);
   if (h->ev_stop) cudaEventDestroy(h->ev_stop);
@@ -831,15 +844,39 @@ seg_status seg_train_step_host_async(seg_handle* h, const void* x_host, const in
                                      float* loss_host) {
   if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
-  const void* x_dev = mapped_device_pointer(x_host);
-  const int32_t* cls_dev = reinterpret_cast<const int32_t*>(mapped_device_pointer(cls_host));
+  if (!mapped_device_pointer(x_host) || !mapped_device_pointer(cls_host)) return SEG_ERR_INVALID_ARG;   // pageable
   float* loss_dev = nullptr;
   if (loss_host) {
     loss_dev = reinterpret_cast<float*>(const_cast<void*>(mapped_device_pointer(loss_host)));
     if (!loss_dev) return SEG_ERR_INVALID_ARG;
   }
-  if (!x_dev || !cls_dev) return SEG_ERR_INVALID_ARG;      // pageable memory cannot be read while the host runs on
-  return seg_train_step(h, x_dev, cls_dev, batch, loss_dev, nullptr);
+  // The batch travels on a copy stream into one of two device buffers, so that the transfer of this
+  // step's batch overlaps the kernels of the steps enqueued before it; the step waits for its copy, and a
+  // buffer is overwritten only after the step that last read it is complete.
+  seg_status st;
+  const size_t row_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
+  if (!h->copy_stream) {
+    SEG_TRY(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking), "copy stream");
+    for (int i = 0; i < 2; ++i) {
+      char* p = nullptr;
+      if ((st = dev_alloc(h, &p, (size_t)h->max_batch * row_bytes, false)) != SEG_OK) return st;
+      h->async_x[i] = p;
+      if ((st = dev_alloc(h, &h->async_cls[i], h->max_batch, false)) != SEG_OK) return st;
+      SEG_TRY(h, cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming), "event create");
+      SEG_TRY(h, cudaEventCreateWithFlags(&h->ev_consumed[i], cudaEventDisableTiming), "event create");
+    }
+  }
+  const int i = h->async_next;
+  h->async_next ^= 1;
+  if (h->async_used[i]) SEG_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_consumed[i], 0), "stream wait");
+  SEG_TRY(h, cudaMemcpyAsync(h->async_x[i], x_host, batch * row_bytes, cudaMemcpyHostToDevice, h->copy_stream), "input copy");
+  SEG_TRY(h, cudaMemcpyAsync(h->async_cls[i], cls_host, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, h->copy_stream), "class copy");
+  SEG_TRY(h, cudaEventRecord(h->ev_copied[i], h->copy_stream), "event record");
+  SEG_TRY(h, cudaStreamWaitEvent(h->stream, h->ev_copied[i], 0), "stream wait");
+  if ((st = seg_train_step(h, h->async_x[i], h->async_cls[i], batch, loss_dev, nullptr)) != SEG_OK) return st;
+  SEG_TRY(h, cudaEventRecord(h->ev_consumed[i], h->stream), "event record");
+  h->async_used[i] = true;
+  return SEG_OK;
 }
 
 seg_status seg_get_labels(seg_handle* h, float* dst) {
