@@ -31,10 +31,11 @@ from paper_2403_11204_b200 import workloads as wl
 
 L2_BYTES = 126 * 1024 * 1024
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel kind, from the
-# ncu capture summarised in profiles/gemm_tc_splitk_paper_shaped.md (forward products of segment 1; average
-# of the three captured launches).  Workloads without a capture of their dominant kind report null.
-NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): 2.26e6}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the product kernel kinds, from the
+# ncu capture summarised in profiles/gemm_traffic_paper_shaped.md (every product launch of two steady-state
+# steps of both segments; mean per kind).  Workloads without a capture of their dominant kind report null.
+NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): 2.600e6, ("paper_shaped", "dgrad_gemm"): 2.952e6,
+                     ("paper_shaped", "wgrad_gemm"): 1.325e6}
 
 
 # ---- peaks -----------------------------------------------------------------------------------
