@@ -400,6 +400,26 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
                                     "stored for the next (seg_train_epochs + seg_forward_dataset)",
                             "samples": n_all, "ms": ms_proc,
                             "samples_per_s": n_all / (ms_proc * 1e-3)}
+    if full and not w.concurrent and len(w.segments) == 2:
+        # recovery phase of Section 5: the left segment trained through the frozen right one, per step
+        from paper_2403_11204_b200 import binding
+        rec_loss = torch.zeros(1, device="cuda")
+        n_rec = max(10, min(steps, 100))
+        for s in range(5):
+            sl = r.batch_slice(s)
+            binding.recovery_step(r.segs[0], r.segs[1], r.x[0][sl], r.cls[sl], rec_loss)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for s in range(n_rec):
+            sl = r.batch_slice(s + 5)
+            binding.recovery_step(r.segs[0], r.segs[1], r.x[0][sl], r.cls[sl], rec_loss)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_rec = e0.elapsed_time(e1) / n_rec
+        out["recovery"] = {"what": "seg_recovery_step: left segment trained through the frozen right segment "
+                                   "(eager launches)", "steps": n_rec, "ms_per_step": ms_rec,
+                           "samples_per_s": w.batch / (ms_rec * 1e-3)}
     r.close()
     del r
     torch.cuda.empty_cache()
@@ -497,7 +517,7 @@ def main():
             "config": config, "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"],
             "roofline": res.get("roofline"), "kernels": res.get("kernels"), "segments": res["segments"],
             "label_gen_ms": res["label_gen_ms"], "memory": res.get("memory"), "procedure": res.get("procedure"),
-            "peaks": peaks}
+            "recovery": res.get("recovery"), "peaks": peaks}
     if not args.no_cpu_baseline:
         line["cpu_baseline"], _ = oracle_samples_per_s(w, budget_s=15.0)
     others = {}

@@ -28,6 +28,8 @@
  *   SEG_NO_GRAPH=1        launch every kernel eagerly instead of replaying a captured step
  *   SEG_NO_FORK=1         run every branch of a step on one stream
  *   SEG_NO_PDL=1          ordinary launches instead of programmatic dependent launches
+ *   SEG_NO_FUSED_LOSS=1   always run the intermediate-label loss as a launch of its own (default: inside
+ *                         the last forward product's epilogue where the tensor-core path can take it)
  *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
  *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
  *   SEG_PAIR_MIN_TILES=n  use CTA pairs exactly when a product has n or more tiles of 256 x 256

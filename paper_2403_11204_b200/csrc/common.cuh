@@ -23,6 +23,27 @@ enum Epilogue : int {
 // Device status word values (written by kernels that give up a bounded wait).
 enum DevStatus : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
 
+// The loss of a non-final segment fused into the epilogue of its last forward product (Section 2:
+// the target is the intermediate label of the sample's class; the final segment's softmax
+// cross-entropy always runs as a launch of its own).  The epilogue still stores the layer's output;
+// in addition it writes dZ of that layer and adds up the batch loss (one partial per CTA; the last
+// CTA to finish adds the partials in index order, writes the loss to the address found in *loss_dst
+// and leaves the counter at zero).
+struct LossFuse {
+  int enabled;              // 0: no fused loss
+  const int32_t* cls;       // [M]: class index of every row
+  const float* sil;         // [classes][N] fp32 targets
+  void* dz;                 // [M][ld_dz] of dz_dt, rounded by dz_round
+  int64_t ld_dz;
+  int dz_dt, dz_round;
+  int relu_mask;            // dZ = 0 where the stored output is not positive
+  float gscale;             // dZ factor: 2/(M N)
+  float loss_scale;         // factor of the summed loss: 1/(M N)
+  float* partials;          // one float per CTA of the launch
+  unsigned int* counter;    // arrival counter, zero between launches
+  float* const* loss_dst;   // device slot holding the address that receives the loss
+};
+
 // One matrix product  C[M][N] = sum_k A(m,k) * B(k,n)  with explicit element strides, so that
 // forward (A W^T), dgrad (dZ W) and wgrad (dZ^T A) are all expressed by one description.
 struct GemmDesc {
@@ -38,6 +59,7 @@ struct GemmDesc {
   const float* bias;        // EPI_BIAS_ACT: [N]
   const void* mask;         // EPI_MASK: [M][ldmask] of c_dt
   int64_t ldmask;
+  LossFuse loss;            // EPI_BIAS_ACT only
   int off_critical_path;    // 1: the product runs beside others (a weight gradient on its branch): the tiling is
                             // chosen for latency plus the SM time it takes away from them, not for latency alone
   // FFMA path only: workspace for splitting K over several CTAs of one tile (may be null: no split).
@@ -55,21 +77,24 @@ int gemm_simt_slots(int M, int N, int K);   // workspace slots (partial 64 x 64 
 // Tensor-core path.  Returns cudaErrorNotSupported when the shape/stride does not fit its TMA rules.
 cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s);
 bool gemm_tc_init();   // resolves the driver entry point needed for tensor maps
+// True when launch_gemm_tc would take the intermediate-label loss into the forward product M x N x K.
+bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32);
 
 cudaError_t launch_gen_labels(float* dst, int n_classes, int n_p, uint64_t seed, int segment_id,
                               int dist, float kappa, cudaStream_t s);
 cudaError_t launch_init_uniform(float* dst, int rows, int cols, int64_t ld, uint64_t seed,
                                 int segment_id, int layer, int tag, float bound, cudaStream_t s);
 
-// loss kernels: write dZ (dz_dt, rounded by dz_round) and a deterministic batch loss
+// loss kernels: write dZ (dz_dt, rounded by dz_round) and a deterministic batch loss, which goes to
+// the address stored in the device slot *loss_dst (the input-staging launch of the step fills it)
 cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const int32_t* cls,
                             const float* sil, int n_p, int batch, int relu_mask,
                             void* dz, int dz_dt, int dz_round, int64_t ld_dz,
-                            float* partials, unsigned int* counter, float* loss_out, cudaStream_t s);
+                            float* partials, unsigned int* counter, float* const* loss_dst, cudaStream_t s);
 cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const int32_t* cls,
                                    int n_classes, int batch, int relu_mask,
                                    void* dz, int dz_dt, int dz_round, int64_t ld_dz,
-                                   float* partials, unsigned int* counter, float* loss_out,
+                                   float* partials, unsigned int* counter, float* const* loss_dst,
                                    cudaStream_t s);
 int loss_max_partials();
 
@@ -100,11 +125,12 @@ cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src
                           int64_t ld_src, int rows, int cols, int round, cudaStream_t s);
 // the same copy plus an int32 vector copy (class indices) in one launch; when t is not null the
 // launch also advances the step counter: t += 1, bc = {1 - beta1^t, 1 - beta2^t}; when gather_src is not
-// null, row r of the destination is row cls[r] of that fp32 [classes][cols] matrix instead of src's row r
+// null, row r of the destination is row cls[r] of that fp32 [classes][cols] matrix instead of src's row r;
+// when loss_dst is not null the launch stores loss_out there (the step's loss kernel reads it back)
 cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2,
-                                const float* gather_src, cudaStream_t s);
+                                const float* gather_src, float* loss_out, float** loss_dst, cudaStream_t s);
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // Kernels of one stream are launched with programmatic stream serialisation: a kernel may become

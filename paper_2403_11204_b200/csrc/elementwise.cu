@@ -41,9 +41,10 @@ __device__ float block_sum(float v, float* smem /* >= 32 floats */) {
 }
 
 // Writes this block's partial; the last block to finish adds all partials in index order and
-// writes loss_out = scale * total.  The counter is left at zero for the next launch.
+// writes scale * total to loss_out, or, when loss_dst is not null, to the address stored in
+// *loss_dst.  The counter is left at zero for the next launch.
 __device__ void finish_loss(float block_total, float* partials, unsigned int* counter,
-                            float* loss_out, float scale, float* smem) {
+                            float* loss_out, float* const* loss_dst, float scale, float* smem) {
   __shared__ bool is_last;
   if (threadIdx.x == 0) {
     partials[blockIdx.x] = block_total;
@@ -58,6 +59,7 @@ __device__ void finish_loss(float block_total, float* partials, unsigned int* co
     for (int i = threadIdx.x; i < (int)gridDim.x; i += blockDim.x) v += __ldcg(partials + i);
     const float total = block_sum(v, smem);
     if (threadIdx.x == 0) {
+      if (loss_dst) loss_out = *loss_dst;
       if (loss_out) *loss_out = total * scale;
       *counter = 0u;
     }
@@ -71,7 +73,7 @@ __global__ void __launch_bounds__(kLossThreads)
 mse_loss_kernel(const TOut* __restrict__ out, int64_t ld_out, const int32_t* __restrict__ cls,
                 const float* __restrict__ sil, int n_p, int batch, int relu_mask,
                 TDz* __restrict__ dz, int dz_round, int64_t ld_dz, float* partials,
-                unsigned int* counter, float* loss_out) {
+                unsigned int* counter, float* loss_out, float* const* loss_dst) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[32];
@@ -94,7 +96,7 @@ mse_loss_kernel(const TOut* __restrict__ out, int64_t ld_out, const int32_t* __r
     else dz[b * ld_dz + i] = g;
   }
   const float bt = block_sum(acc, red);
-  finish_loss(bt, partials, counter, loss_out, 1.0f / (float)total, red);
+  finish_loss(bt, partials, counter, loss_out, loss_dst, 1.0f / (float)total, red);
 }
 
 // Final segment: one warp per sample;  p = softmax(z) with the row maximum subtracted,
@@ -103,7 +105,8 @@ template <typename TDz>
 __global__ void __launch_bounds__(kLossThreads)
 softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* __restrict__ cls,
                   int n_classes, int batch, int relu_mask, TDz* __restrict__ dz, int dz_round,
-                  int64_t ld_dz, float* partials, unsigned int* counter, float* loss_out) {
+                  int64_t ld_dz, float* partials, unsigned int* counter, float* loss_out,
+                  float* const* loss_dst) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[32];
@@ -133,7 +136,7 @@ softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* _
     if (lane == 0) acc += logf(se) - (z[c] - mx);
   }
   const float bt = block_sum(acc, red);
-  finish_loss(bt, partials, counter, loss_out, inv_b, red);
+  finish_loss(bt, partials, counter, loss_out, loss_dst, inv_b, red);
 }
 
 // One optimizer step on one element (Section 3: SGD with momentum; plain SGD and Adam as well).
@@ -263,11 +266,12 @@ copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt
 __global__ void __launch_bounds__(256)
 stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows, int cols,
                     int round, int32_t* cls_dst, const int32_t* cls_src, unsigned long long* t, float* bc,
-                    float beta1, float beta2, const float* gather_src) {
+                    float beta1, float beta2, const float* gather_src, float* loss_out, float** loss_dst) {
   pdl_wait();
   pdl_trigger();
   const int64_t total = (int64_t)rows * cols;
   const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (tid == 0 && loss_dst != nullptr) *loss_dst = loss_out;   // where this step's loss kernel writes the loss
   if (tid == 0 && t != nullptr) {           // step counter and Adam bias corrections of this step
     const unsigned long long step = *t + 1ull;
     *t = step;
@@ -320,16 +324,17 @@ int loss_max_partials() { return kMaxLossBlocks; }
 cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const int32_t* cls,
                             const float* sil, int n_p, int batch, int relu_mask, void* dz,
                             int dz_dt, int dz_round, int64_t ld_dz, float* partials,
-                            unsigned int* counter, float* loss_out, cudaStream_t s) {
+                            unsigned int* counter, float* const* loss_dst, cudaStream_t s) {
+  float* const loss_out = nullptr;
   const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
   if (out_dt == DT_BF16 && dz_dt == DT_BF16) {
     launch_k(mse_loss_kernel<__nv_bfloat16, __nv_bfloat16>, dim3(grid), dim3(kLossThreads), 0, s, 
         (const __nv_bfloat16*)out, ld_out, cls, sil, n_p, batch, relu_mask, (__nv_bfloat16*)dz,
-        dz_round, ld_dz, partials, counter, loss_out);
+        dz_round, ld_dz, partials, counter, loss_out, loss_dst);
   } else if (out_dt == DT_F32 && dz_dt == DT_F32) {
     launch_k(mse_loss_kernel<float, float>, dim3(grid), dim3(kLossThreads), 0, s, 
         (const float*)out, ld_out, cls, sil, n_p, batch, relu_mask, (float*)dz, dz_round, ld_dz,
-        partials, counter, loss_out);
+        partials, counter, loss_out, loss_dst);
   } else {
     return cudaErrorInvalidValue;
   }
@@ -339,17 +344,18 @@ cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const i
 cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const int32_t* cls,
                                    int n_classes, int batch, int relu_mask, void* dz, int dz_dt,
                                    int dz_round, int64_t ld_dz, float* partials,
-                                   unsigned int* counter, float* loss_out, cudaStream_t s) {
+                                   unsigned int* counter, float* const* loss_dst, cudaStream_t s) {
+  float* const loss_out = nullptr;
   const int warps = kLossThreads / 32;
   const int grid = grid_for(batch, warps, kMaxLossBlocks);
   if (dz_dt == DT_BF16) {
     launch_k(softmax_ce_kernel<__nv_bfloat16>, dim3(grid), dim3(kLossThreads), 0, s, 
         logits, ld_logits, cls, n_classes, batch, relu_mask, (__nv_bfloat16*)dz, dz_round, ld_dz,
-        partials, counter, loss_out);
+        partials, counter, loss_out, loss_dst);
   } else {
     launch_k(softmax_ce_kernel<float>, dim3(grid), dim3(kLossThreads), 0, s, logits, ld_logits, cls, n_classes,
                                                           batch, relu_mask, (float*)dz, dz_round,
-                                                          ld_dz, partials, counter, loss_out);
+                                                          ld_dz, partials, counter, loss_out, loss_dst);
   }
   return cudaGetLastError();
 }
@@ -377,11 +383,11 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
 cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2,
-                                const float* gather_src, cudaStream_t s) {
+                                const float* gather_src, float* loss_out, float** loss_dst, cudaStream_t s) {
   const int esz = dt == DT_BF16 ? 2 : 4;
   const int grid = grid_for((int64_t)rows * cols * esz / 16, 256, 148 * 8);   // one 16-byte group per thread and pass
   launch_k(stage_inputs_kernel, dim3(grid), dim3(256), 0, s, dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
-                                           beta1, beta2, gather_src);
+                                           beta1, beta2, gather_src, loss_out, loss_dst);
   return cudaGetLastError();
 }
 
@@ -449,7 +455,7 @@ extern "C" SEG_API seg_status seg_label_loss_noalloc(const float* out, const int
   if (cudaMemsetAsync(counter, 0, sizeof(unsigned int), s) != cudaSuccess) { cudaGetLastError(); return SEG_ERR_CUDA; }
   const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
   mse_loss_kernel<float, float><<<grid, kLossThreads, 0, s>>>(out, n_p, cls, sil, n_p, batch, relu_mask ? 1 : 0, dz,
-                                                             RND_NONE, n_p, partials, counter, loss_out);
+                                                             RND_NONE, n_p, partials, counter, loss_out, nullptr);
   if (cudaGetLastError() != cudaSuccess) return SEG_ERR_CUDA;
   return SEG_OK;
 }

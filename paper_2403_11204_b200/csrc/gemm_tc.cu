@@ -172,6 +172,7 @@ struct EpilogueArgs {
   const float* bias;
   const void* mask;
   int64_t ldmask;
+  LossFuse loss;
 };
 
 template <int BLOCK_N>
@@ -249,10 +250,9 @@ __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide
 // Columns are stored in groups of 8 with 16-byte accesses when the group count is whole and the
 // row segment is 16-byte aligned (every lane touches its own row, so wide accesses are what keeps
 // the number of memory wavefronts down); ragged or unaligned segments fall back to scalar stores.
-__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], const EpiSide& s, int row,
-                                               int col0, int n_total) {
+__device__ __forceinline__ void epilogue_values(const EpilogueArgs& e, float (&v)[32], const EpiSide& s, int col0,
+                                                int n_total) {
   const int n_valid = min(32, n_total - col0);
-  const bool whole = (n_valid & 7) == 0;
   if (e.epi == EPI_BIAS_ACT) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __uint_as_float(s.w[j]);
@@ -278,8 +278,15 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = round_tf32_rne(v[j]);
   }
-  if (e.c_dt == DT_BF16) {
-    __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(e.C) + (int64_t)row * e.ldc + col0;
+}
+
+// Stores up to 32 consecutive columns of one row into a [rows][ld] matrix of dtype dt.
+__device__ __forceinline__ void store_row_segment(void* base, int dt, int64_t ld, const float (&v)[32], int row,
+                                                  int col0, int n_total) {
+  const int n_valid = min(32, n_total - col0);
+  const bool whole = (n_valid & 7) == 0;
+  if (dt == DT_BF16) {
+    __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(base) + (int64_t)row * ld + col0;
     if (whole && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
 #pragma unroll
       for (int j = 0; j < 32; j += 8) {
@@ -299,7 +306,7 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
       for (int j = 0; j < 32; ++j) if (j < n_valid) crow[j] = __float2bfloat16_rn(v[j]);
     }
   } else {
-    float* crow = reinterpret_cast<float*>(e.C) + (int64_t)row * e.ldc + col0;
+    float* crow = reinterpret_cast<float*>(base) + (int64_t)row * ld + col0;
     if (whole && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
 #pragma unroll
       for (int j = 0; j < 32; j += 4) {
@@ -312,7 +319,98 @@ __device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)
   }
 }
 
-template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
+__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], const EpiSide& s, int row,
+                                               int col0, int n_total) {
+  epilogue_values(e, v, s, col0, n_total);
+  store_row_segment(e.C, e.c_dt, e.ldc, v, row, col0, n_total);
+}
+
+// ---- fused loss (last forward product of a non-final segment) -----------------------------------
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// Targets of n_cols (<= 32) consecutive columns of one row: row cls[row] of the label matrix, whose
+// pitch is n_p.  Fetched ahead of the accumulator like the other side inputs.
+__device__ __forceinline__ void loss_prefetch_target(const LossFuse& l, EpiSide& t, int row, bool row_ok, int col0,
+                                                     int n_cols, int n_p) {
+  if (n_cols <= 0 || !row_ok) return;
+  const float* trow = l.sil + (int64_t)__ldg(l.cls + row) * n_p + col0;
+  if (((n_cols & 3) == 0) && ((reinterpret_cast<uintptr_t>(trow) & 15u) == 0)) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      if (j < n_cols) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(trow + j));
+        t.w[j] = q.x; t.w[j + 1] = q.y; t.w[j + 2] = q.z; t.w[j + 3] = q.w;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) if (j < n_cols) t.w[j] = __float_as_uint(__ldg(trow + j));
+  }
+}
+
+// Mean-squared-error part of the epilogue for columns [col0, n_end): stores the output, then
+// dZ = gscale (a - t) [a > 0], and adds (a - t)^2 to the thread's loss sum; a is the output as it
+// is stored (after rounding to the storage type).
+__device__ __forceinline__ void epilogue_store_mse(const EpilogueArgs& e, float (&v)[32], const EpiSide& s,
+                                                   const EpiSide& t, int row, int col0, int n_end, float& lacc) {
+  epilogue_values(e, v, s, col0, n_end);
+  store_row_segment(e.C, e.c_dt, e.ldc, v, row, col0, n_end);
+  const int n_valid = min(32, n_end - col0);
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    if (j < n_valid) {
+      const float a = (e.c_dt == DT_BF16) ? round_bf16_rne(v[j]) : v[j];
+      const float d = a - __uint_as_float(t.w[j]);
+      lacc = fmaf(d, d, lacc);
+      float g = d * e.loss.gscale;
+      if (e.loss.relu_mask && !(a > 0.f)) g = 0.f;
+      v[j] = apply_round(g, e.loss.dz_round);
+    }
+  }
+  store_row_segment(e.loss.dz, e.loss.dz_dt, e.loss.ld_dz, v, row, col0, n_end);
+}
+
+// End of a CTA's epilogue: the four epilogue warps leave their loss sums in shared memory; the last
+// warp to arrive adds them in warp order and publishes the CTA's partial; the last CTA of the grid
+// adds all partials in index order (a fixed order: bit-reproducible) and writes the batch loss.
+// No barrier is used, so a warp that gave up a bounded wait cannot block the others.
+__device__ __forceinline__ void loss_finish(const LossFuse& l, float lacc, int quarter, int lane, volatile float* slots,
+                                            unsigned int* warp_counter) {
+  const float w = warp_sum_f(lacc);
+  unsigned int prev = 0;
+  if (lane == 0) {
+    slots[quarter] = w;
+    __threadfence_block();
+    prev = atomicAdd(warp_counter, 1u);
+  }
+  prev = __shfl_sync(0xFFFFFFFFu, prev, 0);
+  if (prev != 3u) return;
+  __threadfence_block();
+  unsigned int done = 0;
+  if (lane == 0) {
+    const float block_total = ((slots[0] + slots[1]) + slots[2]) + slots[3];
+    l.partials[blockIdx.x] = block_total;
+    __threadfence();
+    done = atomicAdd(l.counter, 1u);
+  }
+  done = __shfl_sync(0xFFFFFFFFu, done, 0);
+  if (done != gridDim.x - 1) return;
+  __threadfence();
+  float part = 0.f;
+  for (unsigned int i = lane; i < gridDim.x; i += 32) part += __ldcg(l.partials + i);
+  const float total = warp_sum_f(part);
+  if (lane == 0) {
+    float* dst = *l.loss_dst;
+    if (dst) *dst = total * l.loss_scale;
+    *l.counter = 0u;
+  }
+}
+
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N, bool LOSS = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                int M, int N, int K, EpilogueArgs epi, int* dev_status) {
@@ -332,6 +430,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile float* loss_slots = reinterpret_cast<volatile float*>(reinterpret_cast<uint8_t*>(bars) + 256);
+  unsigned int* loss_warps = reinterpret_cast<unsigned int*>(reinterpret_cast<uint8_t*>(bars) + 272);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar_base = smem_u32(bars);
@@ -346,6 +446,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     *abort_flag = 0;
+    *loss_warps = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -438,27 +539,39 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. +31 belong to this warp
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
+    float lacc = 0.f;                      // LOSS: this thread's share of the batch loss
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
       const int m0 = (t % tiles_m) * BLOCK_M, n0 = (t / tiles_m) * BLOCK_N;
       const int row = m0 + quarter * 32 + lane;
-      EpiSide side, side_next;
+      EpiSide side, side_next, tgt, tgt_next;
       epilogue_prefetch(epi, side, row, row < M, n0, N);   // before the wait: latency off the critical path
+      if constexpr (LOSS) loss_prefetch_target(epi.loss, tgt, row, row < M, n0, min(32, N - n0), N);
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= N) break;              // uniform across the CTA
-        if (c + 1 < BLOCK_N / 32) epilogue_prefetch(epi, side_next, row, row < M, col0 + 32, N);
+        if (c + 1 < BLOCK_N / 32) {
+          epilogue_prefetch(epi, side_next, row, row < M, col0 + 32, N);
+          if constexpr (LOSS) loss_prefetch_target(epi.loss, tgt_next, row, row < M, col0 + 32, min(32, N - col0 - 32), N);
+        }
         float v[32];
         tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
-        if (row < M) epilogue_store(epi, v, side, row, col0, N);
+        if (row < M) {
+          if constexpr (LOSS) epilogue_store_mse(epi, v, side, tgt, row, col0, N, lacc);
+          else epilogue_store(epi, v, side, row, col0, N);
+        }
         side = side_next;
+        if constexpr (LOSS) tgt = tgt_next;
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+    if constexpr (LOSS) {
+      if (ok) loss_finish(epi.loss, lacc, quarter, lane, loss_slots, loss_warps);
     }
   }
 
@@ -498,7 +611,7 @@ constexpr int SPLITK_RECV_BYTES = 8 * (SPLITK_BLOCK_N / 8) * BLOCK_M * 4;       
 constexpr int SPLITK_SMEM = SPLITK_STAGES * SPLITK_STAGE_BYTES + 2 * SPLITK_RECV_BYTES + SMEM_EXTRA;   // + send buffer
 
 // One 128 x 64 output tile per cluster; CTA r of the cluster contracts k-blocks [r*kpc, (r+1)*kpc).
-template <bool TF32, bool A_MN, bool B_MN>
+template <bool TF32, bool A_MN, bool B_MN, bool LOSS = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                       int M, int N, int K, int split, EpilogueArgs epi, int* dev_status) {
@@ -521,6 +634,8 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   // bars[0..S) full, [S..2S) empty, [2S] accumulator complete, [2S+1] partial slices received
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile float* loss_slots = reinterpret_cast<volatile float*>(reinterpret_cast<uint8_t*>(bars) + 256);
+  unsigned int* loss_warps = reinterpret_cast<unsigned int*>(reinterpret_cast<uint8_t*>(bars) + 272);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -537,6 +652,7 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     mbar_init(acc_bar, 1);
     mbar_init(recv_bar, 1);
     *abort_flag = 0;
+    *loss_warps = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     // this CTA will receive one column slice (BLOCK_N / split columns x 128 rows, fp32) from every peer
@@ -624,8 +740,10 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     const int row = m0 + row_in_tile;
     const int w = BLOCK_N / split;                         // columns owned by each CTA: 32, 16 or 8
     const int own_col0 = n0 + (int)rank * w;
-    EpiSide side;                                          // side inputs of this CTA's slice, fetched ahead
+    EpiSide side, tgt;                                     // side inputs of this CTA's slice, fetched ahead
     epilogue_prefetch(epi, side, row, row < M, own_col0, min(N, own_col0 + w));
+    if constexpr (LOSS) loss_prefetch_target(epi.loss, tgt, row, row < M, own_col0, min(w, N - own_col0), N);
+    float lacc = 0.f;
     bool ok = mbar_wait(acc_bar, 0, abort_flag, dev_status);
     tc_fence_after();
     const uint32_t slice_bytes = (uint32_t)(w * BLOCK_M * 4);
@@ -672,7 +790,11 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         for (int cs = 0; cs < 32; ++cs)
           if (cs < w) own[cs] += recv[(src * w + cs) * BLOCK_M + row_in_tile];
       }
-      if (row < M && own_col0 < N) epilogue_store(epi, own, side, row, own_col0, min(N, own_col0 + w));
+      if (row < M && own_col0 < N) {
+        if constexpr (LOSS) epilogue_store_mse(epi, own, side, tgt, row, own_col0, min(N, own_col0 + w), lacc);
+        else epilogue_store(epi, own, side, row, own_col0, min(N, own_col0 + w));
+      }
+      if constexpr (LOSS) loss_finish(epi.loss, lacc, quarter, lane, loss_slots, loss_warps);
     }
     tc_fence_before();
   }
@@ -941,11 +1063,11 @@ bool make_map(CUtensorMap* map, bool f32, const void* base, uint64_t inner, uint
   return r == CUDA_SUCCESS;
 }
 
-template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N, bool LOSS = false>
 cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                            const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   using L = SmemLayout<BLOCK_N>;
-  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N>;
+  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N, LOSS>;
   static bool attr_set_dev[64] = {};      // the attribute is per device
   bool& attr_set = attr_set_dev[current_device_slot()];
   if (!attr_set) {
@@ -961,17 +1083,20 @@ cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const G
 template <bool TF32, int BLOCK_N>
 cudaError_t launch_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUtensorMap& mb,
                           const GemmDesc& g, const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
-  if (!a_mn && !b_mn) return launch_variant<TF32, false, false, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  if (!a_mn && !b_mn) {
+    if (e.loss.enabled) return launch_variant<TF32, false, false, BLOCK_N, true>(ma, mb, g, e, dev_status, s);
+    return launch_variant<TF32, false, false, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  }
   if (!a_mn && b_mn) return launch_variant<TF32, false, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
   if (a_mn && b_mn) return launch_variant<TF32, true, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
   return cudaErrorNotSupported;
 }
 
 
-template <bool TF32, bool A_MN, bool B_MN>
+template <bool TF32, bool A_MN, bool B_MN, bool LOSS = false>
 cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                                   const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
-  auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN>;
+  auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN, LOSS>;
   static bool attr_set_dev[64] = {};      // the attribute is per device
   bool& attr_set = attr_set_dev[current_device_slot()];
   if (!attr_set) {
@@ -997,7 +1122,10 @@ cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, 
 template <bool TF32>
 cudaError_t launch_splitk_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUtensorMap& mb,
                                  const GemmDesc& g, const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
-  if (!a_mn && !b_mn) return launch_splitk_variant<TF32, false, false>(ma, mb, g, e, split, dev_status, s);
+  if (!a_mn && !b_mn) {
+    if (e.loss.enabled) return launch_splitk_variant<TF32, false, false, true>(ma, mb, g, e, split, dev_status, s);
+    return launch_splitk_variant<TF32, false, false>(ma, mb, g, e, split, dev_status, s);
+  }
   if (!a_mn && b_mn) return launch_splitk_variant<TF32, false, true>(ma, mb, g, e, split, dev_status, s);
   if (a_mn && b_mn) return launch_splitk_variant<TF32, true, true>(ma, mb, g, e, split, dev_status, s);
   return cudaErrorNotSupported;
@@ -1122,6 +1250,18 @@ bool gemm_tc_init() {
   return g_init_ok;
 }
 
+// The mean-squared-error loss of a non-final segment is fused into the single-CTA and split-K kernels.
+// The CTA-pair kernel serves large products, where a separate loss launch costs next to nothing.
+// Softmax cross-entropy was tried in the epilogue (one thread per row of at most 64 logits) and
+// measured 3-4 times slower than the separate warp-per-row kernel: long straight-line code that every
+// thread runs once.
+bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32) {
+  if (!g_init_ok) return false;
+  const int split = g_allow_splitk ? pick_split(M, N, K, tf32) : 1;
+  if (split > 1) return true;
+  return pick_kernel(M, N, K, tf32, false).kind == 0;
+}
+
 cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   if (!g_init_ok) return cudaErrorNotSupported;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return cudaErrorNotSupported;
@@ -1143,6 +1283,9 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   if ((a_pitch * esz) % 16 != 0 || (b_pitch * esz) % 16 != 0) return cudaErrorNotSupported;
   if (a_pitch * (int64_t)esz >= (1ll << 40) || b_pitch * (int64_t)esz >= (1ll << 40)) return cudaErrorNotSupported;
 
+  const bool fuse_loss = (g.epi == EPI_BIAS_ACT) && g.loss.enabled != 0;
+  if (fuse_loss && (a_mn || b_mn || !gemm_tc_can_fuse_loss(g.M, g.N, g.K, tf32)))
+    return cudaErrorInvalidValue;                           // the caller asks gemm_tc_can_fuse_loss first
   const bool throughput = g.off_critical_path != 0;
   const int split = (g_allow_splitk && !throughput) ? pick_split(g.M, g.N, g.K, tf32) : 1;
   const Choice choice = pick_kernel(g.M, g.N, g.K, tf32, throughput);
@@ -1161,6 +1304,7 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   EpilogueArgs e;
   e.C = g.C; e.ldc = g.ldc; e.c_dt = g.c_dt; e.c_round = g.c_round; e.epi = g.epi; e.relu = g.relu;
   e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
+  e.loss = g.loss; e.loss.enabled = fuse_loss ? 1 : 0;
 
   if (pairs) {
     return tf32 ? launch_pair_majors<true>(a_mn, b_mn, ma, mb, g, e, dev_status, s)

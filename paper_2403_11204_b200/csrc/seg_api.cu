@@ -70,6 +70,7 @@ struct seg_handle {
   int32_t* cls_stage = nullptr;
   std::vector<void*> dzbuf;        // index 0..L-1
   float* loss_slot = nullptr;
+  float** loss_dst = nullptr;      // device slot: where the current step's loss goes (filled by the staging launch)
   unsigned long long* step_dev = nullptr;
   float* bc_dev = nullptr;
   // FFMA path: split-K workspaces.  Index 0 serves the main branch (its products run one after another),
@@ -80,23 +81,24 @@ struct seg_handle {
   std::vector<cudaStream_t> lstream;  // lstream[l], l >= 1: the branch of layer l (weight gradient, then update)
   std::vector<cudaEvent_t> ev_dz;     // ev_dz[l]: dZ_l is complete (main branch)
   std::vector<cudaEvent_t> ev_done;   // ev_done[l], l >= 1: layer l's branch is complete
-  // A captured step.  The caller's pointers enter the graph in two kernel nodes only (input staging:
-  // x and cls; loss: loss_out); their parameters are rewritten before every replay.
+  // A captured step.  The caller's pointers (x, cls, loss_out) enter the graph in one kernel node only,
+  // the input staging; its parameters are rewritten before a replay when they differ.
   struct StepGraph {
     int eager_runs = 0;
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
     uint64_t kernels = 0;
-    cudaGraphNode_t stage_node = nullptr, loss_node = nullptr;
-    cudaKernelNodeParams stage_params{}, loss_params{};
-    std::vector<void*> stage_args, loss_args;
+    cudaGraphNode_t stage_node = nullptr;
+    cudaKernelNodeParams stage_params{};
+    std::vector<void*> stage_args;
     const void* cur_x = nullptr; const int32_t* cur_cls = nullptr; float* cur_loss = nullptr;   // now in the exec
     const float* cur_gather = nullptr;
   };
-  cudaGraphNode_t cap_stage_node = nullptr, cap_loss_node = nullptr;   // filled while capturing
+  cudaGraphNode_t cap_stage_node = nullptr;   // filled while capturing
   bool capturing = false;
   std::map<int, StepGraph> graphs; // by batch size
   bool graphs_enabled = true;
+  bool fuse_loss = true;           // take the intermediate-label loss in the last forward product's epilogue where possible
   bool fork_enabled = true;        // run the gradient and update branches on their own streams
   float* sil = nullptr;
   bool have_labels = false;
@@ -223,8 +225,44 @@ seg_status prepare_input(seg_handle* h, const void* x, int batch, const void** x
   return SEG_OK;
 }
 
-// Forward products of all layers, reading layer 0's input from (a_prev, ld_prev).
-seg_status forward_layers(seg_handle* h, const void* a_prev, int64_t ld_prev, int batch) {
+// Description of a non-final segment's loss for fusion into its last forward product.
+LossFuse loss_fuse_desc(seg_handle* h, int batch, const int32_t* cls, float* const* loss_dst) {
+  const int L = h->n_layers;
+  LossFuse f{};
+  f.enabled = 1;
+  f.cls = cls; f.sil = h->sil;
+  f.dz = h->dzbuf[L - 1]; f.ld_dz = h->ld_act[L]; f.dz_dt = h->act_dt; f.dz_round = h->act_round;
+  f.relu_mask = h->last_relu ? 1 : 0;
+  const double count = (double)batch * h->widths[L];
+  f.gscale = 2.0f / (float)((int64_t)batch * h->widths[L]);
+  f.loss_scale = (float)(1.0 / count);
+  f.partials = h->loss_partials; f.counter = h->loss_counter; f.loss_dst = loss_dst;
+  return f;
+}
+
+// The segment's loss as a launch of its own (the final segment's softmax cross-entropy always; the
+// intermediate-label loss when the last forward product could not take it).
+seg_status launch_loss(seg_handle* h, int batch, const int32_t* cls, float* const* loss_dst) {
+  const int L = h->n_layers;
+  Launch l(h, K_LOSS, h->stream);
+  void* dz_L = h->dzbuf[L - 1];
+  if (h->is_final) {
+    SEG_TRY(h, launch_softmax_ce_loss((const float*)h->act[L], h->ld_act[L], cls, h->n_classes, batch,
+                                      h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
+                                      h->loss_partials, h->loss_counter, loss_dst, h->stream), "softmax-CE loss");
+  } else {
+    SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], cls, h->sil, h->widths[L], batch,
+                               h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
+                               h->loss_partials, h->loss_counter, loss_dst, h->stream), "MSE loss");
+  }
+  return SEG_OK;
+}
+
+// Forward products of all layers, reading layer 0's input from (a_prev, ld_prev).  With loss_cls not
+// null the segment's loss follows: inside the last product's epilogue where the tensor-core path can
+// take it, as a separate launch otherwise.
+seg_status forward_layers(seg_handle* h, const void* a_prev, int64_t ld_prev, int batch,
+                          const int32_t* loss_cls = nullptr, float* const* loss_dst = nullptr) {
   for (int l = 0; l < h->n_layers; ++l) {
     const LayerInfo& L = h->layers[l];
     const bool last = (l == h->n_layers - 1);
@@ -236,8 +274,14 @@ seg_status forward_layers(seg_handle* h, const void* a_prev, int64_t ld_prev, in
     g.c_round = (last && h->is_final) ? RND_NONE : h->act_round;
     g.epi = EPI_BIAS_ACT; g.relu = (!last || h->last_relu) ? 1 : 0;
     g.bias = h->params + L.b_off;
-    seg_status st = run_gemm(h, g, K_FWD, h->stream);
+    const bool want_loss = last && loss_cls != nullptr;
+    if (want_loss && !h->is_final && h->use_tc && h->fuse_loss &&
+        gemm_tc_can_fuse_loss(g.M, g.N, g.K, h->precision == SEG_TF32))
+      g.loss = loss_fuse_desc(h, batch, loss_cls, loss_dst);
+    bool used_tc = false;
+    seg_status st = run_gemm(h, g, K_FWD, h->stream, &used_tc);
     if (st != SEG_OK) return st;
+    if (want_loss && !(used_tc && g.loss.enabled) && (st = launch_loss(h, batch, loss_cls, loss_dst)) != SEG_OK) return st;
     a_prev = h->act[l + 1]; ld_prev = h->ld_act[l + 1];
   }
   h->last_batch = batch;
@@ -380,6 +424,7 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   }
   if ((st = dev_alloc(h, &h->cls_stage, h->max_batch, true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->loss_slot, 1, true)) != SEG_OK) return bail(st);
+  if ((st = dev_alloc(h, &h->loss_dst, 1, true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->step_dev, 1, true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->bc_dev, 2, true)) != SEG_OK) return bail(st);
   h->lstream.assign(h->n_layers, nullptr);
@@ -397,6 +442,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
     if (env && env[0] == '1') g_use_pdl = false;
     env = getenv("SEG_NO_FORK");
     if (env && env[0] == '1') h->fork_enabled = false;
+    env = getenv("SEG_NO_FUSED_LOSS");
+    if (env && env[0] == '1') h->fuse_loss = false;
   }
   if (!h->use_tc) {
     // split-K workspaces of the FFMA path, sized for the products each one serves at max_batch
@@ -506,34 +553,20 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked);
 
 static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void* x, const int32_t* cls,
                                float* loss_out, const float* gather) {
-  const int L = h->n_layers;
   cudaStream_t mainst = h->stream;
   seg_status st;
-  float* loss_dst = loss_out ? loss_out : h->loss_slot;
+  float* loss_to = loss_out ? loss_out : h->loss_slot;
   {
     // fixed staging buffers: rounds x in TF32 mode, pads the pitch, keeps every later pointer constant;
-    // the same launch advances the device-side step counter and Adam's bias corrections
+    // the same launch advances the device-side step counter and Adam's bias corrections and records
+    // where this step's loss goes
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   gather, mainst), "input staging");
+                                   gather, loss_to, h->loss_dst, mainst), "input staging");
   }
   if (h->capturing) h->cap_stage_node = last_captured_node(h);
-  if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
-  {
-    Launch l(h, K_LOSS, mainst);
-    void* dz_L = h->dzbuf[L - 1];
-    if (h->is_final) {
-      SEG_TRY(h, launch_softmax_ce_loss((const float*)h->act[L], h->ld_act[L], h->cls_stage, h->n_classes, batch,
-                                        h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
-                                        h->loss_partials, h->loss_counter, loss_dst, mainst), "softmax-CE loss");
-    } else {
-      SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], h->cls_stage, h->sil, h->widths[L], batch,
-                                 h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
-                                 h->loss_partials, h->loss_counter, loss_dst, mainst), "MSE loss");
-    }
-  }
-  if (h->capturing) h->cap_loss_node = last_captured_node(h);
+  if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch, h->cls_stage, h->loss_dst)) != SEG_OK) return st;
   return enqueue_backward(h, batch, forked);
 }
 
@@ -601,16 +634,13 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
 }
 
 // Index of the caller-supplied pointers in the kernels' parameter lists (see elementwise.cu).
-static const int kStageArgCount = 15, kStageArgX = 3, kStageArgCls = 9, kStageArgGather = 14;
-static int loss_arg_count(const seg_handle* h) { return h->is_final ? 12 : 13; }
+static const int kStageArgCount = 17, kStageArgX = 3, kStageArgCls = 9, kStageArgGather = 14, kStageArgLoss = 15;
 
 static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGraph_t graph) {
-  if (!h->cap_stage_node || !h->cap_loss_node) return false;
-  g.stage_node = h->cap_stage_node; g.loss_node = h->cap_loss_node;
+  if (!h->cap_stage_node) return false;
+  g.stage_node = h->cap_stage_node;
   if (cudaGraphKernelNodeGetParams(g.stage_node, &g.stage_params) != cudaSuccess) return false;
-  if (cudaGraphKernelNodeGetParams(g.loss_node, &g.loss_params) != cudaSuccess) return false;
   g.stage_args.assign(g.stage_params.kernelParams, g.stage_params.kernelParams + kStageArgCount);
-  g.loss_args.assign(g.loss_params.kernelParams, g.loss_params.kernelParams + loss_arg_count(h));
   if (cudaGraphInstantiate(&g.exec, graph, 0) != cudaSuccess) { g.exec = nullptr; return false; }
   g.graph = graph;                      // kept alive: the parameter blocks above belong to it
   return true;
@@ -618,22 +648,16 @@ static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGr
 
 static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const void* x, const int32_t* cls,
                                float* loss_out, const float* gather) {
-  float* loss_dst = loss_out ? loss_out : h->loss_slot;
-  if (x != g.cur_x || cls != g.cur_cls || gather != g.cur_gather) {
+  float* loss_to = loss_out ? loss_out : h->loss_slot;
+  if (x != g.cur_x || cls != g.cur_cls || gather != g.cur_gather || loss_to != g.cur_loss) {
     g.stage_args[kStageArgX] = (void*)&x;
     g.stage_args[kStageArgCls] = (void*)&cls;
     g.stage_args[kStageArgGather] = (void*)&gather;
+    g.stage_args[kStageArgLoss] = (void*)&loss_to;
     cudaKernelNodeParams sp = g.stage_params;
     sp.kernelParams = g.stage_args.data();
     SEG_TRY(h, cudaGraphExecKernelNodeSetParams(g.exec, g.stage_node, &sp), "graph parameter update");
-    g.cur_x = x; g.cur_cls = cls; g.cur_gather = gather;
-  }
-  if (loss_dst != g.cur_loss) {
-    g.loss_args[loss_arg_count(h) - 1] = (void*)&loss_dst;
-    cudaKernelNodeParams lp = g.loss_params;
-    lp.kernelParams = g.loss_args.data();
-    SEG_TRY(h, cudaGraphExecKernelNodeSetParams(g.exec, g.loss_node, &lp), "graph parameter update");
-    g.cur_loss = loss_dst;
+    g.cur_x = x; g.cur_cls = cls; g.cur_gather = gather; g.cur_loss = loss_to;
   }
   SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
   h->launches += g.kernels;
@@ -679,7 +703,7 @@ static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* c
         h->graphs_enabled = false;
         st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
       } else {
-        h->capturing = true; h->cap_stage_node = nullptr; h->cap_loss_node = nullptr;
+        h->capturing = true; h->cap_stage_node = nullptr;
         st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
         h->capturing = false;
         cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
@@ -690,9 +714,8 @@ static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* c
         } else {
           // capture did not work here: run eagerly from now on
           if (getenv("SEG_DEBUG"))
-            fprintf(stderr, "seg: step capture failed (status %d, end-capture '%s', nodes %p %p, last '%s')\n", (int)st,
-                    cudaGetErrorString(e), (void*)h->cap_stage_node, (void*)h->cap_loss_node,
-                    cudaGetErrorString(cudaPeekAtLastError()));
+            fprintf(stderr, "seg: step capture failed (status %d, end-capture '%s', node %p, last '%s')\n", (int)st,
+                    cudaGetErrorString(e), (void*)h->cap_stage_node, cudaGetErrorString(cudaPeekAtLastError()));
           cudaGetLastError();
           if (graph) cudaGraphDestroy(graph);
           g.exec = nullptr;
@@ -726,17 +749,11 @@ seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x,
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   nullptr, s), "input staging");
+                                   nullptr, loss_out ? loss_out : r->loss_slot, h->loss_dst, s), "input staging");
   }
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
-  if ((st = forward_layers(r, h->act[Ll], h->ld_act[Ll], batch)) != SEG_OK) return st;
-  {
-    Launch l(r, K_LOSS, s);
-    SEG_TRY(r, launch_softmax_ce_loss((const float*)r->act[Lr], r->ld_act[Lr], h->cls_stage, r->n_classes, batch,
-                                      r->last_relu ? 1 : 0, r->dzbuf[Lr - 1], r->act_dt, r->act_round, r->ld_act[Lr],
-                                      r->loss_partials, r->loss_counter, loss_out ? loss_out : r->loss_slot, s),
-            "softmax-CE loss");
-  }
+  // the joined network's loss: the right segment's softmax cross-entropy on the class labels
+  if ((st = forward_layers(r, h->act[Ll], h->ld_act[Ll], batch, h->cls_stage, h->loss_dst)) != SEG_OK) return st;
   // through the frozen right segment: dgrad only, down to its input, which is the left segment's output
   for (int l = Lr - 1; l >= 0; --l) {
     const LayerInfo& Ly = r->layers[l];

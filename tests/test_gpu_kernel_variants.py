@@ -2,7 +2,9 @@
 small problems, CTA pairs for large ones).  The small parity shapes would never reach the CTA-pair
 kernel or the unsplit kernel on their own, so the tensor-core parity cases are run again in child
 processes with the selection forced through the library's environment switches (read once per
-process, hence the child processes)."""
+process, hence the child processes).  The same goes for the intermediate-label loss, which the
+tensor-core path takes inside the last forward product's epilogue: SEG_NO_FUSED_LOSS runs the separate
+loss kernel."""
 import os
 import subprocess
 import sys
@@ -14,7 +16,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 @pytest.mark.parametrize("env", [{"SEG_PAIR_MIN_TILES": "1"}, {"SEG_NO_SPLITK": "1", "SEG_NO_PAIRS": "1"},
-                                 {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}, {"SEG_NO_PDL": "1"}])
+                                 {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}, {"SEG_NO_PDL": "1"},
+                                 {"SEG_NO_FUSED_LOSS": "1"}])
 def test_tensor_core_cases_with_forced_kernel_selection(env):
     child_env = dict(os.environ, **env)
     res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",
