@@ -277,6 +277,13 @@ def unpartitioned_comparison(workload, steps=5):
     return {"layers": len(widths) - 1, "mem_bytes_peak": mem, "ms_per_step": ms}
 
 
+def _rank_barrier():
+    """Barrier over the replicas when the run has more than one (a no-op otherwise)."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
 def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples=None):
     """Runs one workload.  full=True adds the end-to-end leg, per-kernel profile and clocks."""
     import torch
@@ -296,7 +303,9 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
         sampler.start()
         time.sleep(0.25)
     l0 = r.launches()
-    ms = r.timed(warmup, steps)
+    _rank_barrier()                       # replicas start the timed region together ...
+    ms = r.timed(warmup, steps)           # (synchronises the device on both sides; CUDA events on every stream)
+    _rank_barrier()                       # ... and leave it together
     launches = r.launches() - l0
     if full:
         time.sleep(0.15)
