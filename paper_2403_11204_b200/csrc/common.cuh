@@ -23,12 +23,12 @@ enum Epilogue : int {
 // Device status word values (written by kernels that give up a bounded wait).
 enum DevStatus : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
 
-// The loss of a non-final segment fused into the epilogue of its last forward product (Section 2:
-// the target is the intermediate label of the sample's class; the final segment's softmax
-// cross-entropy always runs as a launch of its own).  The epilogue still stores the layer's output;
-// in addition it writes dZ of that layer and adds up the batch loss (one partial per CTA; the last
-// CTA to finish adds the partials in index order, writes the loss to the address found in *loss_dst
-// and leaves the counter at zero).
+// The loss of a non-final segment fused into the epilogue of its last forward product when the
+// split-K kernel runs it (Section 2: the target is the intermediate label of the sample's class; the
+// final segment's softmax cross-entropy always runs as a launch of its own).  The epilogue still
+// stores the layer's output; in addition it writes dZ of that layer and adds up the batch loss (one
+// partial per CTA; the last CTA to finish adds the partials in index order, writes the loss to the
+// address found in *loss_dst and leaves the counter at zero).
 struct LossFuse {
   int enabled;              // 0: no fused loss
   const int32_t* cls;       // [M]: class index of every row

@@ -410,7 +410,7 @@ __device__ __forceinline__ void loss_finish(const LossFuse& l, float lacc, int q
   }
 }
 
-template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N, bool LOSS = false>
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                int M, int N, int K, EpilogueArgs epi, int* dev_status) {
@@ -430,8 +430,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile float* loss_slots = reinterpret_cast<volatile float*>(reinterpret_cast<uint8_t*>(bars) + 256);
-  unsigned int* loss_warps = reinterpret_cast<unsigned int*>(reinterpret_cast<uint8_t*>(bars) + 272);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar_base = smem_u32(bars);
@@ -446,7 +444,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     *abort_flag = 0;
-    *loss_warps = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -539,39 +536,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. +31 belong to this warp
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
-    float lacc = 0.f;                      // LOSS: this thread's share of the batch loss
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
       const int m0 = (t % tiles_m) * BLOCK_M, n0 = (t / tiles_m) * BLOCK_N;
       const int row = m0 + quarter * 32 + lane;
-      EpiSide side, side_next, tgt, tgt_next;
+      EpiSide side, side_next;
       epilogue_prefetch(epi, side, row, row < M, n0, N);   // before the wait: latency off the critical path
-      if constexpr (LOSS) loss_prefetch_target(epi.loss, tgt, row, row < M, n0, min(32, N - n0), N);
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= N) break;              // uniform across the CTA
-        if (c + 1 < BLOCK_N / 32) {
-          epilogue_prefetch(epi, side_next, row, row < M, col0 + 32, N);
-          if constexpr (LOSS) loss_prefetch_target(epi.loss, tgt_next, row, row < M, col0 + 32, min(32, N - col0 - 32), N);
-        }
+        if (c + 1 < BLOCK_N / 32) epilogue_prefetch(epi, side_next, row, row < M, col0 + 32, N);
         float v[32];
         tmem_load_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
-        if (row < M) {
-          if constexpr (LOSS) epilogue_store_mse(epi, v, side, tgt, row, col0, N, lacc);
-          else epilogue_store(epi, v, side, row, col0, N);
-        }
+        if (row < M) epilogue_store(epi, v, side, row, col0, N);
         side = side_next;
-        if constexpr (LOSS) tgt = tgt_next;
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-    }
-    if constexpr (LOSS) {
-      if (ok) loss_finish(epi.loss, lacc, quarter, lane, loss_slots, loss_warps);
     }
   }
 
@@ -1063,11 +1048,11 @@ bool make_map(CUtensorMap* map, bool f32, const void* base, uint64_t inner, uint
   return r == CUDA_SUCCESS;
 }
 
-template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N, bool LOSS = false>
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
 cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                            const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   using L = SmemLayout<BLOCK_N>;
-  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N, LOSS>;
+  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N>;
   static bool attr_set_dev[64] = {};      // the attribute is per device
   bool& attr_set = attr_set_dev[current_device_slot()];
   if (!attr_set) {
@@ -1083,10 +1068,7 @@ cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const G
 template <bool TF32, int BLOCK_N>
 cudaError_t launch_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUtensorMap& mb,
                           const GemmDesc& g, const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
-  if (!a_mn && !b_mn) {
-    if (e.loss.enabled) return launch_variant<TF32, false, false, BLOCK_N, true>(ma, mb, g, e, dev_status, s);
-    return launch_variant<TF32, false, false, BLOCK_N>(ma, mb, g, e, dev_status, s);
-  }
+  if (!a_mn && !b_mn) return launch_variant<TF32, false, false, BLOCK_N>(ma, mb, g, e, dev_status, s);
   if (!a_mn && b_mn) return launch_variant<TF32, false, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
   if (a_mn && b_mn) return launch_variant<TF32, true, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
   return cudaErrorNotSupported;
@@ -1250,16 +1232,16 @@ bool gemm_tc_init() {
   return g_init_ok;
 }
 
-// The mean-squared-error loss of a non-final segment is fused into the single-CTA and split-K kernels.
-// The CTA-pair kernel serves large products, where a separate loss launch costs next to nothing.
-// Softmax cross-entropy was tried in the epilogue (one thread per row of at most 64 logits) and
-// measured 3-4 times slower than the separate warp-per-row kernel: long straight-line code that every
-// thread runs once.
+// The mean-squared-error loss of a non-final segment is fused into the split-K kernel, the one that
+// serves the small, latency-bound products: there it replaces a launch on the critical path for about
+// 3 us of extra epilogue (paper_shaped: -3 us per step).  In the single-CTA kernel of mid-sized
+// products the same epilogue measured slower than the separate loss launch (bf16_wide 1024x2048x4096:
+// 44 us against 25 + 14 us under ncu), and the CTA-pair kernel serves large products, where a separate
+// loss launch costs next to nothing.  Softmax cross-entropy was tried in the epilogue as well (one
+// thread per row of at most 64 logits) and measured 3-4 times slower than the warp-per-row kernel.
 bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32) {
-  if (!g_init_ok) return false;
-  const int split = g_allow_splitk ? pick_split(M, N, K, tf32) : 1;
-  if (split > 1) return true;
-  return pick_kernel(M, N, K, tf32, false).kind == 0;
+  if (!g_init_ok || !g_allow_splitk) return false;
+  return pick_split(M, N, K, tf32) > 1;
 }
 
 cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
