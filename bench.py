@@ -34,8 +34,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the product kernel kinds, from the
 # ncu capture summarised in profiles/gemm_traffic_paper_shaped.md (every product launch of two steady-state
 # steps of both segments; mean per kind).  Workloads without a capture of their dominant kind report null.
-NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): 2.600e6, ("paper_shaped", "dgrad_gemm"): 2.952e6,
-                     ("paper_shaped", "wgrad_gemm"): 1.325e6}
+NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): 2.621e6, ("paper_shaped", "dgrad_gemm"): 2.953e6,
+                     ("paper_shaped", "wgrad_gemm"): 1.326e6}
 
 
 # ---- peaks -----------------------------------------------------------------------------------
