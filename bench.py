@@ -427,7 +427,7 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
         torch.cuda.synchronize()
         ms_rec = e0.elapsed_time(e1) / n_rec
         out["recovery"] = {"what": "seg_recovery_step: left segment trained through the frozen right segment "
-                                   "(eager launches)", "steps": n_rec, "ms_per_step": ms_rec,
+                                   "(one replayed graph per step)", "steps": n_rec, "ms_per_step": ms_rec,
                            "samples_per_s": w.batch / (ms_rec * 1e-3)}
     r.close()
     del r

@@ -26,6 +26,7 @@
 #include <stdlib.h>
 
 #include <algorithm>
+#include <functional>
 #include <map>
 #include <new>
 #include <string>
@@ -87,7 +88,8 @@ struct seg_handle {
     int eager_runs = 0;
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
-    uint64_t kernels = 0;
+    uint64_t kernels = 0, kernels_peer = 0;
+    seg_handle* peer = nullptr;
     cudaGraphNode_t stage_node = nullptr;
     cudaKernelNodeParams stage_params{};
     std::vector<void*> stage_args;
@@ -97,6 +99,8 @@ struct seg_handle {
   cudaGraphNode_t cap_stage_node = nullptr;   // filled while capturing
   bool capturing = false;
   std::map<int, StepGraph> graphs; // by batch size
+  std::map<std::pair<uint64_t, int>, StepGraph> recovery_graphs;   // by (right segment's uid, batch size)
+  uint64_t uid = 0;                // unique per handle of the process (a reused address is not the same segment)
   bool graphs_enabled = true;
   bool fuse_loss = true;           // take the intermediate-label loss in the last forward product's epilogue where possible
   bool fork_enabled = true;        // run the gradient and update branches on their own streams
@@ -360,6 +364,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
 
   seg_handle* h = new (std::nothrow) seg_handle();
   if (!h) return SEG_ERR_ALLOC;
+  static uint64_t next_uid = 0;
+  h->uid = ++next_uid;
   h->n_layers = cfg->n_layers; h->n_classes = cfg->n_classes; h->max_batch = cfg->max_batch;
   h->segment_id = cfg->segment_id; h->is_final = cfg->is_final != 0;
   h->last_relu = cfg->last_relu < 0 ? !h->is_final : (cfg->last_relu != 0);
@@ -494,6 +500,10 @@ seg_status seg_destroy(seg_handle* h) {
   cudaStreamSynchronize(h->stream);
   for (cudaStream_t ls : h->lstream) if (ls) cudaStreamSynchronize(ls);
   for (auto& kv : h->graphs) {
+    if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+    if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
+  }
+  for (auto& kv : h->recovery_graphs) {
     if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
     if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
   }
@@ -647,8 +657,7 @@ static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGr
 }
 
 static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const void* x, const int32_t* cls,
-                               float* loss_out, const float* gather) {
-  float* loss_to = loss_out ? loss_out : h->loss_slot;
+                               float* loss_to, const float* gather) {
   if (x != g.cur_x || cls != g.cur_cls || gather != g.cur_gather || loss_to != g.cur_loss) {
     g.stage_args[kStageArgX] = (void*)&x;
     g.stage_args[kStageArgCls] = (void*)&cls;
@@ -661,7 +670,51 @@ static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const vo
   }
   SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
   h->launches += g.kernels;
+  if (g.peer) g.peer->launches += g.kernels_peer;
   return SEG_OK;
+}
+
+// Runs one step through its captured graph: the first call with this graph slot runs eagerly (it sets
+// kernel attributes), the second captures the same enqueue into a graph, later ones replay it with the
+// caller's pointers written into the staging node.  enqueue(forked) enqueues the whole step; peer is a
+// second handle whose kernels the step launches (the frozen right segment of a recovery step) or null.
+static seg_status run_step_captured(seg_handle* h, seg_handle::StepGraph& g, seg_handle* peer,
+                                    const std::function<seg_status(bool)>& enqueue,
+                                    const void* x, const int32_t* cls, float* loss_to, const float* gather) {
+  if (g.exec != nullptr) return replay_graph(h, g, x, cls, loss_to, gather);
+  if (g.eager_runs == 0) {
+    g.eager_runs = 1;
+    return enqueue(h->fork_enabled);
+  }
+  const uint64_t before = h->launches, before_peer = peer ? peer->launches : 0;
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    h->graphs_enabled = false;
+    return enqueue(h->fork_enabled);
+  }
+  h->capturing = true; h->cap_stage_node = nullptr;
+  seg_status st = enqueue(h->fork_enabled);
+  h->capturing = false;
+  cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
+  if (st == SEG_OK && e == cudaSuccess && graph != nullptr && adopt_captured_graph(h, g, graph)) {
+    g.kernels = h->launches - before;
+    h->launches = before;
+    g.peer = peer;
+    if (peer) { g.kernels_peer = peer->launches - before_peer; peer->launches = before_peer; }
+    return replay_graph(h, g, x, cls, loss_to, gather);
+  }
+  // capture did not work here: run eagerly from now on
+  if (getenv("SEG_DEBUG"))
+    fprintf(stderr, "seg: step capture failed (status %d, end-capture '%s', node %p, last '%s')\n", (int)st,
+            cudaGetErrorString(e), (void*)h->cap_stage_node, cudaGetErrorString(cudaPeekAtLastError()));
+  cudaGetLastError();
+  if (graph) cudaGraphDestroy(graph);
+  g.exec = nullptr;
+  h->graphs_enabled = false;
+  h->launches = before;
+  if (peer) peer->launches = before_peer;
+  return enqueue(h->fork_enabled);
 }
 
 static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
@@ -689,42 +742,8 @@ static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* c
   if (h->profile || !h->graphs_enabled) {
     st = enqueue_step(h, batch, !h->profile && h->fork_enabled, x, cls, loss_out, gather);
   } else {
-    seg_handle::StepGraph& g = h->graphs[batch];
-    if (g.exec != nullptr) {
-      st = replay_graph(h, g, x, cls, loss_out, gather);
-    } else if (g.eager_runs == 0) {
-      st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);   // first step at this batch size: eager (sets kernel attributes)
-      g.eager_runs = 1;
-    } else {
-      const uint64_t before = h->launches;
-      cudaGraph_t graph = nullptr;
-      if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-        cudaGetLastError();
-        h->graphs_enabled = false;
-        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
-      } else {
-        h->capturing = true; h->cap_stage_node = nullptr;
-        st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
-        h->capturing = false;
-        cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
-        if (st == SEG_OK && e == cudaSuccess && graph != nullptr && adopt_captured_graph(h, g, graph)) {
-          g.kernels = h->launches - before;
-          h->launches = before;
-          st = replay_graph(h, g, x, cls, loss_out, gather);
-        } else {
-          // capture did not work here: run eagerly from now on
-          if (getenv("SEG_DEBUG"))
-            fprintf(stderr, "seg: step capture failed (status %d, end-capture '%s', node %p, last '%s')\n", (int)st,
-                    cudaGetErrorString(e), (void*)h->cap_stage_node, cudaGetErrorString(cudaPeekAtLastError()));
-          cudaGetLastError();
-          if (graph) cudaGraphDestroy(graph);
-          g.exec = nullptr;
-          h->graphs_enabled = false;
-          h->launches = before;
-          st = enqueue_step(h, batch, h->fork_enabled, x, cls, loss_out, gather);
-        }
-      }
-    }
+    auto enqueue = [&](bool forked) { return enqueue_step(h, batch, forked, x, cls, loss_out, gather); };
+    st = run_step_captured(h, h->graphs[batch], nullptr, enqueue, x, cls, loss_out ? loss_out : h->loss_slot, gather);
   }
   if (st != SEG_OK) return st;
   ++h->step;
@@ -733,15 +752,8 @@ static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* c
 }
 
 // Recovery step (Section 5 of the paper): the left segment keeps training through the frozen right one.
-seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x, const int32_t* cls,
-                             int32_t batch, float* loss_out) {
-  if (!left || !right || !x || !cls) return SEG_ERR_INVALID_ARG;
-  if (batch < 1 || batch > left->max_batch || batch > right->max_batch) return SEG_ERR_SHAPE;
-  if (left->is_final || !right->is_final) return SEG_ERR_STATE;
-  if (left->widths[left->n_layers] != right->widths[0]) return SEG_ERR_SHAPE;
-  if (left->precision != right->precision || left->stream != right->stream) return SEG_ERR_UNSUPPORTED;
-  seg_handle* h = left;
-  seg_handle* r = right;
+static seg_status enqueue_recovery(seg_handle* h, seg_handle* r, int batch, bool forked, const void* x,
+                                   const int32_t* cls, float* loss_to) {
   const int Ll = h->n_layers, Lr = r->n_layers;
   cudaStream_t s = h->stream;
   seg_status st;
@@ -749,8 +761,9 @@ seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x,
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   nullptr, loss_out ? loss_out : r->loss_slot, h->loss_dst, s), "input staging");
+                                   nullptr, loss_to, h->loss_dst, s), "input staging");
   }
+  if (h->capturing) h->cap_stage_node = last_captured_node(h);
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
   // the joined network's loss: the right segment's softmax cross-entropy on the class labels
   if ((st = forward_layers(r, h->act[Ll], h->ld_act[Ll], batch, h->cls_stage, h->loss_dst)) != SEG_OK) return st;
@@ -771,8 +784,31 @@ seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x,
     }
     if ((st = run_gemm(r, d, K_DGRAD, s)) != SEG_OK) return st;
   }
-  if ((st = enqueue_backward(h, batch, !h->profile && h->fork_enabled)) != SEG_OK) return st;
+  return enqueue_backward(h, batch, forked);
+}
+
+seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x, const int32_t* cls,
+                             int32_t batch, float* loss_out) {
+  if (!left || !right || !x || !cls) return SEG_ERR_INVALID_ARG;
+  if (batch < 1 || batch > left->max_batch || batch > right->max_batch) return SEG_ERR_SHAPE;
+  if (left->is_final || !right->is_final) return SEG_ERR_STATE;
+  if (left->widths[left->n_layers] != right->widths[0]) return SEG_ERR_SHAPE;
+  if (left->precision != right->precision || left->stream != right->stream) return SEG_ERR_UNSUPPORTED;
+  seg_handle* h = left;
+  seg_handle* r = right;
+  float* loss_to = loss_out ? loss_out : r->loss_slot;
+  seg_status st;
+  if (h->profile || r->profile || !h->graphs_enabled) {
+    st = enqueue_recovery(h, r, batch, !h->profile && !r->profile && h->fork_enabled, x, cls, loss_to);
+  } else {
+    // captured like an ordinary step; the graph holds the right segment's buffers, so it is keyed by that
+    // segment's identity and dropped with the left handle
+    auto enqueue = [&](bool forked) { return enqueue_recovery(h, r, batch, forked, x, cls, loss_to); };
+    st = run_step_captured(h, h->recovery_graphs[std::make_pair(r->uid, (int)batch)], r, enqueue, x, cls, loss_to, nullptr);
+  }
+  if (st != SEG_OK) return st;
   ++h->step;
+  h->last_batch = r->last_batch = batch;
   return SEG_OK;
 }
 

@@ -57,12 +57,14 @@ def test_recovery_step_matches_the_oracle(precision, backend, tol):
     x, cls = batch_arrays(w, batch, 784, precision=precision)
     xt, ct = to_device(x, cls, precision)
     right_before = [t.clone() for l in range(2) for t in gr.params(l)]
-    for step in range(2):
+    for step in range(4):                                   # eager, captured, replayed twice
         loss_t = torch.zeros(1, device="cuda")
         binding.recovery_step(gl, gr, xt, ct, loss_t)
         gl.poll()
         loss_o = pnn.recovery_step(ol, orr, x, cls.astype(np.int64))
         assert abs(float(loss_t.item()) - loss_o) <= tol * abs(loss_o)
+        if step >= 2:
+            continue          # two trajectories in reduced precision drift apart: later steps are held to the loss only
         for l in range(2):
             dW, db = gl.grads(l)
             assert rel_err(dW.cpu().numpy(), ol.dW[l]) <= tol and rel_err(db.cpu().numpy(), ol.db[l]) <= tol
