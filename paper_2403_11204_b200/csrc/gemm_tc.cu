@@ -1237,8 +1237,12 @@ bool gemm_tc_init() {
 // 3 us of extra epilogue (paper_shaped: -3 us per step).  In the single-CTA kernel of mid-sized
 // products the same epilogue measured slower than the separate loss launch (bf16_wide 1024x2048x4096:
 // 44 us against 25 + 14 us under ncu), and the CTA-pair kernel serves large products, where a separate
-// loss launch costs next to nothing.  Softmax cross-entropy was tried in the epilogue as well (one
-// thread per row of at most 64 logits) and measured 3-4 times slower than the warp-per-row kernel.
+// loss launch costs next to nothing.  Softmax cross-entropy was tried in the epilogue of the single-CTA
+// kernel in three forms - one thread per row of at most 64 logits unrolled in registers (3-4 times slower
+// than the separate warp-per-row kernel), the tile left in shared memory with each warp walking its 32
+// rows, lanes over the classes (slower still: 32 dependent reduction chains per warp), and one thread
+// per row with short loops over its row in shared memory (about the cost of the launch it saves, and
+// it gives up the split over K) - and stays a launch of its own.
 bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32) {
   if (!g_init_ok || !g_allow_splitk) return false;
   return pick_split(M, N, K, tf32) > 1;
