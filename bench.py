@@ -8,13 +8,18 @@ workload (forward, loss against the intermediate labels or the class labels, bac
 Intermediate labels are generated once per cut before the timed region, as in the method (the
 label matrix is produced once per training run); that launch is timed separately.
 
-Prints ONE JSON line.  `value` is timed with CUDA events with every input resident in HBM; `e2e`
-goes through the host-buffer entry point (pinned host batches, loss read back every step);
-`roofline` describes the kernel kind with the largest share of the step; `cpu_baseline` is the
-CPU oracle timed on this machine's host cores on a bounded sample.
+The headline workload is the largest one, `gemm_large` (both segments in flight on two streams, the
+second one fed the first cut's label rows by class, i.e. the fully separate variant).  The timed
+region is K steps between CUDA events on every stream in use; it is repeated (at least five times
+and until half a second of device time has been spent) and the MEDIAN repeat is reported, all
+repeats being listed.  Prints ONE JSON line.  `value` has every input resident in HBM; `e2e` goes
+through the host-buffer entry point (pinned host batches in, loss out, every step); `roofline`
+describes the kernel kind with the largest share of the step, timed with CUDA events around every
+launch; `cpu_baseline` is the CPU oracle on this machine's host cores on a bounded sample.
 """
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -31,11 +36,17 @@ from paper_2403_11204_b200 import workloads as wl
 
 L2_BYTES = 126 * 1024 * 1024
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the product kernel kinds, from the
-# ncu capture summarised in profiles/gemm_traffic_paper_shaped.md (every product launch of two steady-state
-# steps of both segments; mean per kind).  Workloads without a capture of their dominant kind report null.
-NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): 2.621e6, ("paper_shaped", "dgrad_gemm"): 2.953e6,
-                     ("paper_shaped", "wgrad_gemm"): 1.326e6}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of product kernels, from the ncu captures
+# summarised under profiles/ (the file named beside each figure).  Workloads without a capture of their dominant
+# kind report null.
+NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): (2.621e6, "profiles/gemm_traffic_paper_shaped.md"),
+                     ("paper_shaped", "dgrad_gemm"): (2.953e6, "profiles/gemm_traffic_paper_shaped.md"),
+                     ("paper_shaped", "wgrad_gemm"): (1.326e6, "profiles/gemm_traffic_paper_shaped.md")}
+
+# Rows per oracle step in the CPU legs (full layer widths always): the oracle converts and rounds every weight
+# matrix at each use, so a step of the largest segments costs seconds whatever the batch.
+CPU_SAMPLE_BATCH = {"tiny": 64, "paper_net": 1410, "paper_shaped": 256, "bf16_wide": 256, "multi_cut": 128,
+                    "gemm_large": 64}
 
 
 # ---- peaks -----------------------------------------------------------------------------------
@@ -46,6 +57,55 @@ def load_peaks():
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
                 "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def measure_tf32_peak(peaks):
+    """TF32 dense peak, measured the way the bf16 figure of MEASURED_PEAKS.json was: torch.matmul on 8192^3
+    with TF32 allowed, best of 10 (burst) and back to back for about a second (sustained).  A library product
+    used as a yardstick only."""
+    import torch
+    try:
+        old = torch.backends.cuda.matmul.allow_tf32
+        torch.backends.cuda.matmul.allow_tf32 = True
+        n = 8192
+        a = torch.randn(n, n, device="cuda")
+        b = torch.randn(n, n, device="cuda")
+        flops = 2.0 * n ** 3
+        for _ in range(3):
+            a @ b
+        best = 0.0
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); a @ b; e1.record()
+            torch.cuda.synchronize()
+            best = max(best, flops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+        reps = max(10, int(1.0 / (flops / (best * 1e12))))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            a @ b
+        e1.record()
+        torch.cuda.synchronize()
+        sustained = reps * flops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+        torch.backends.cuda.matmul.allow_tf32 = old
+        del a, b
+        torch.cuda.empty_cache()
+        peaks["tf32_tflops"], peaks["tf32_tflops_sustained"] = best, sustained
+        peaks["tf32_source"] = "measured in this run: torch.matmul 8192^3 with TF32 allowed, best of 10 / back to back 1 s"
+    except Exception as exc:                                   # keep the nominal ratio, and say so
+        peaks["tf32_tflops"] = 0.5 * peaks["bf16_tflops"]
+        peaks["tf32_tflops_sustained"] = 0.5 * peaks["bf16_tflops_sustained"]
+        peaks["tf32_source"] = f"0.5 x bf16 (nominal ratio; measurement failed: {repr(exc)[:80]})"
+
+
+def tensor_peak_tflops(precision, peaks, sustained=False):
+    """Roofline denominator of the products: the burst figure (the machine's measured peak); the sustained one
+    (a long library product under the power cap) is reported beside it."""
+    if precision == "tf32":
+        if "tf32_tflops" not in peaks:
+            measure_tf32_peak(peaks)
+        return peaks["tf32_tflops_sustained" if sustained else "tf32_tflops"]
+    return peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
 
 
 # ---- algorithmic work --------------------------------------------------------------------------
@@ -67,15 +127,21 @@ def segment_work(spec, batch, precision, optimizer):
             "params": p_w + p_b}
 
 
-def tensor_peak_tflops(precision, peaks, sustained=True):
-    base = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-    return base * (0.5 if precision in ("tf32",) else 1.0)     # nominal TF32 : bf16 ratio is 1 : 2
+def step_fractions(work, ms, precision, peaks):
+    """The two fractions of a (segment) step: the roofline sum (product FLOPs at the tensor peak plus update
+    and loss bytes at the copy bandwidth) over the measured time, and the tensor-only one."""
+    tp = tensor_peak_tflops(precision, peaks)
+    tps = tensor_peak_tflops(precision, peaks, sustained=True)
+    t_roof = work["gemm_flops"] / (tp * 1e12) + (work["update_bytes"] + work["loss_bytes"]) / (peaks["hbm_gbs"] * 1e9)
+    tf = work["gemm_flops"] / (ms * 1e-3) / 1e12
+    return {"roofline_ms": t_roof * 1e3, "roofline_frac": t_roof * 1e3 / ms, "gemm_tflops": tf,
+            "tensor_only_frac": tf / tp, "tensor_only_frac_of_sustained_matmul": tf / tps}
 
 
 # ---- clocks ------------------------------------------------------------------------------------
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index=0):
         self.rows, self.proc, self.index = [], None, index
@@ -102,17 +168,21 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        num = lambda s: s.replace(".", "").isdigit()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and num(r[0])]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and num(r[1])]
+        pw = [float(r[6]) for r in self.rows if len(r) >= 7 and num(r[6])]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(len(r) >= 6 and r[2 + i].lower() == "active" for r in self.rows)]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[2 + i].lower() == "active" for r in self.rows)]
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+                "reasons": reasons, "samples": len(sm), "sm_mhz_min": min(sm) if sm else None,
+                "power_w_max": max(pw) if pw else None}
 
 
 # ---- the CPU oracle leg --------------------------------------------------------------------------
-def oracle_samples_per_s(workload, budget_s=20.0, max_steps=50):
-    """Times the oracle's training step of every segment on batches of the workload."""
+def oracle_samples_per_s(workload, budget_s=20.0, max_steps=50, warmup=0):
+    """Times the oracle's training step of every segment on a bounded sample of the workload: full layer
+    widths, CPU_SAMPLE_BATCH rows per step (the workload's own batch where that is no larger)."""
     from oracle import rng as orng
     from oracle.segment import OracleSegment
     try:
@@ -121,6 +191,7 @@ def oracle_samples_per_s(workload, budget_s=20.0, max_steps=50):
     except Exception:
         cores = len(os.sched_getaffinity(0))
     w = workload
+    rows = min(w.batch, CPU_SAMPLE_BATCH.get(w.name, w.batch))
     segs = []
     for spec in w.segments:
         s = OracleSegment(spec.widths, w.n_classes, spec.is_final, precision=w.precision, optimizer=w.optimizer,
@@ -128,8 +199,11 @@ def oracle_samples_per_s(workload, budget_s=20.0, max_steps=50):
         if not spec.is_final:
             s.gen_labels(wl.LABEL_SEED, orng.DIST_NORMAL if w.label_dist == "normal" else orng.DIST_UNIFORM_KAPPA)
         segs.append(s)
-    cls = wl.class_indices(w, w.batch)
-    xs = [wl.features(w, w.batch, spec.widths[0], seed=spec.segment_id) for spec in w.segments]
+    cls = wl.class_indices(w, rows)
+    xs = [wl.features(w, rows, spec.widths[0], seed=spec.segment_id) for spec in w.segments]
+    for _ in range(warmup):
+        for s, x in zip(segs, xs):
+            s.train_step(x, cls)
     t_total, steps = 0.0, 0
     while steps < max_steps and (t_total < budget_s or steps < 1):
         t0 = time.perf_counter()
@@ -137,9 +211,10 @@ def oracle_samples_per_s(workload, budget_s=20.0, max_steps=50):
             s.train_step(x, cls)
         t_total += time.perf_counter() - t0
         steps += 1
-    return {"value": steps * w.batch / t_total, "unit": "samples/s", "cores": cores, "kind": "oracle",
-            "sample": f"{steps} full-shape step(s) of every segment at batch {w.batch} "
-                      f"({t_total:.1f} s of NumPy fp64 on the host cores)"}, t_total / steps
+    what = "full-shape" if rows == w.batch else f"full-width, {rows}-row (of the workload's {w.batch})"
+    return {"value": steps * rows / t_total, "unit": "samples/s", "cores": cores, "kind": "oracle",
+            "sample": f"{steps} {what} step(s) of every segment ({t_total:.1f} s of NumPy fp64 on the host cores; "
+                      f"samples/s = rows / time, the per-step cost of converting the weights included)"}, t_total / steps
 
 
 # ---- our arm -----------------------------------------------------------------------------------
@@ -180,6 +255,7 @@ class Runner:
                 x = torch.rand(self.n, n_feat, generator=g, device="cuda", dtype=torch.float32)
             self.x = [x.to(self.dt)]
             self.cls = torch.randint(0, w.n_classes, (self.n,), generator=g, device="cuda", dtype=torch.int32)
+        self.sil_in = [None] * len(self.segs)
         torch.cuda.synchronize()
 
     def gen_labels(self):
@@ -192,16 +268,20 @@ class Runner:
 
     def materialise_inputs(self):
         """Inputs of segment k > 0: the stored response of segment k-1 over the whole set (Section 2).
-        For concurrently trained segments the input is the label row of each sample's class."""
+        Concurrently trained segments take the label row of each sample's class instead (the fully separate
+        variant): nothing is materialised, seg_train_step_label_input gathers the rows inside the step."""
         torch, w = self.torch, self.w
         for k in range(1, len(self.segs)):
             prev = self.segs[k - 1]
             if w.concurrent:
-                xk = prev.labels()[self.cls.long()].to(self.dt).contiguous()
-            else:
-                xk = torch.empty(self.n, prev.widths[-1], dtype=prev.out_dtype, device="cuda")
-                for i in range(0, self.n, w.batch):
-                    prev.forward(self.x[k - 1][i:i + w.batch], xk[i:i + w.batch])
+                self.sil_in[k] = prev.labels()
+                self.x.append(None)
+                if self.host_x is not None:
+                    self.host_x.append(None)
+                continue
+            xk = torch.empty(self.n, prev.widths[-1], dtype=prev.out_dtype, device="cuda")
+            for i in range(0, self.n, w.batch):
+                prev.forward(self.x[k - 1][i:i + w.batch], xk[i:i + w.batch])
             self.x.append(xk)
             if self.host_x is not None:
                 self.host_x.append(xk.cpu().pin_memory())
@@ -211,13 +291,19 @@ class Runner:
         i = (step * self.w.batch) % self.n
         return slice(i, i + self.w.batch)
 
+    def step_segment(self, k, sl):
+        seg = self.segs[k]
+        if self.sil_in[k] is not None:
+            seg.train_step_label_input(self.sil_in[k], self.cls[sl], self.loss[k])
+        else:
+            seg.train_step(self.x[k][sl], self.cls[sl], self.loss[k])
+
     def run_steps(self, first, count, which=None):
         for s in range(first, first + count):
             sl = self.batch_slice(s)
-            for k, seg in enumerate(self.segs):
-                if which is not None and k != which:
-                    continue
-                seg.train_step(self.x[k][sl], self.cls[sl], self.loss[k])
+            for k in range(len(self.segs)):
+                if which is None or k == which:
+                    self.step_segment(k, sl)
 
     def timed(self, first, count, which=None):
         """Device time of `count` steps (ms): CUDA events on every stream in use, max over streams."""
@@ -242,6 +328,13 @@ class Runner:
 
     def launches(self):
         return sum(seg.launch_count() for seg in self.segs)
+
+    def families(self):
+        out = {}
+        for seg in self.segs:
+            for name, n in seg.product_launches().items():
+                out[name] = out.get(name, 0) + n
+        return out
 
     def close(self):
         for seg in self.segs:
@@ -284,8 +377,68 @@ def _rank_barrier():
         dist.barrier()
 
 
-def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples=None):
-    """Runs one workload.  full=True adds the end-to-end leg, per-kernel profile and clocks."""
+def kernel_breakdown(r, steps, first, peaks):
+    """Per-kind device time: the same steps again with CUDA events around every launch (one stream, so the
+    kinds add up to the serial time of a step).  Returns (kernels dict, roofline dict of the dominant kind)."""
+    w = r.w
+    for seg in r.segs:
+        seg.profile(True)
+    r.run_steps(first, steps)
+    r.torch.cuda.synchronize()
+    kinds = {}
+    for spec, seg in zip(w.segments, r.segs):
+        work = segment_work(spec, w.batch, w.precision, w.optimizer)
+        for name, (n, tot) in seg.profile_read().items():
+            k = kinds.setdefault(name, {"launches": 0, "ms": 0.0, "flops": 0.0, "bytes": 0.0})
+            k["launches"] += n
+            k["ms"] += tot
+            if name in ("fwd_gemm", "dgrad_gemm", "wgrad_gemm"):
+                k["flops"] += work[name] * steps
+            elif name == "update":          # the update launch also reads dZ for the bias gradient
+                k["bytes"] += (work["update_bytes"] + work["bias_grad_bytes"]) * steps
+            elif name == "loss":
+                k["bytes"] += work["loss_bytes"] * steps
+        seg.profile(False)
+    tp = tensor_peak_tflops(w.precision, peaks)
+    tps = tensor_peak_tflops(w.precision, peaks, sustained=True)
+    total_ms = sum(v["ms"] for v in kinds.values()) or 1.0
+    kernels = {}
+    for n, v in kinds.items():
+        if v["launches"] == 0:
+            continue
+        e = {"launches": v["launches"], "ms_per_step": round(v["ms"] / steps, 5), "share": round(v["ms"] / total_ms, 4),
+             "avg_us": round(1e3 * v["ms"] / v["launches"], 3)}
+        if v["flops"] > 0:
+            e["tflops"] = round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2)
+            e["frac_of_peak"] = round(e["tflops"] / tp, 4)
+        elif v["bytes"] > 0:
+            e["gbs"] = round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1)
+            e["frac_of_peak"] = round(e["gbs"] / peaks["hbm_gbs"], 4)
+        kernels[n] = e
+    dom = max(kinds, key=lambda n: kinds[n]["ms"])
+    v = kinds[dom]
+    timing = "CUDA events around every launch of this kind on the launching stream, same steps re-run after the timed region"
+    traffic = NCU_TRAFFIC_BYTES.get((w.name, dom))
+    if v["flops"] > 0:
+        achieved = v["flops"] / (v["ms"] * 1e-3) / 1e12
+        prec_note = (peaks.get("tf32_source", "") if w.precision == "tf32" else "bf16 torch.matmul burst figure")
+        roof = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": tp, "unit": "TFLOP/s",
+                "frac": achieved / tp, "frac_of_sustained_matmul": achieved / tps, "peak_sustained": tps,
+                "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
+                "peak_source": f"{peaks['source']} ({prec_note})", "timing": timing,
+                "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
+    else:
+        achieved = v["bytes"] / (v["ms"] * 1e-3) / 1e9
+        roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                "peak_source": f"{peaks['source']}: copy bandwidth", "timing": timing,
+                "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
+    return kernels, roof
+
+
+def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples=None, extras=False):
+    """Runs one workload.  full=True adds the end-to-end leg and the clock record; extras=True the training
+    procedure and recovery legs (two sequential segments)."""
     import torch
     w = workload
     if n_samples is None and not full:
@@ -294,7 +447,7 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
     r.prepare()
     label_ms = r.gen_labels()
     r.materialise_inputs()
-    data_bytes = sum(x.numel() * x.element_size() for x in r.x)
+    data_bytes = sum(x.numel() * x.element_size() for x in r.x if x is not None)
     r.run_steps(0, max(warmup, 3))
     for seg in r.segs:
         seg.poll()
@@ -302,86 +455,79 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
     if full:
         sampler.start()
         time.sleep(0.25)
-    l0 = r.launches()
-    _rank_barrier()                       # replicas start the timed region together ...
-    ms = r.timed(warmup, steps)           # (synchronises the device on both sides; CUDA events on every stream)
-    _rank_barrier()                       # ... and leave it together
+    # the timed region, repeated: exactly `steps` steps per repeat, at least 5 repeats and 0.5 s of device time
+    l0, f0 = r.launches(), r.families()
+    repeats, total_ms, pos = [], 0.0, warmup
+    min_repeats, max_repeats = (5, 400) if full else (3, 20)
+    while len(repeats) < min_repeats or (total_ms < (500.0 if full else 50.0) and len(repeats) < max_repeats):
+        _rank_barrier()                       # replicas enter and leave every timed region together
+        ms = r.timed(pos, steps)              # synchronises the device on both sides; CUDA events on every stream
+        _rank_barrier()
+        repeats.append(ms)
+        total_ms += ms
+        pos += steps
     launches = r.launches() - l0
+    f1 = r.families()
     if full:
         time.sleep(0.15)
     clocks = sampler.stop() if full else None
+    ms = float(np.median(repeats))
     out = {"ms_per_step": ms / steps, "samples_per_s": steps * w.batch / (ms * 1e-3), "launches": launches,
+           "repeats": {"n": len(repeats), "steps_each": steps, "ms_per_step_median": ms / steps,
+                       "ms_per_step_min": min(repeats) / steps, "ms_per_step_max": max(repeats) / steps,
+                       "device_s_total": total_ms * 1e-3},
+           "product_launches": {k: f1[k] - f0.get(k, 0) for k in f1},
            "label_gen_ms": label_ms, "data_bytes": data_bytes, "clocks": clocks, "segments": []}
 
-    # per-segment timing and roofline of the whole segment step
-    tp = tensor_peak_tflops(w.precision, peaks)
+    # per-segment timing (each segment alone on its stream) and the two fractions of the whole segment step
+    whole = {"gemm_flops": 0, "update_bytes": 0, "loss_bytes": 0}
     for k, (spec, seg) in enumerate(zip(w.segments, r.segs)):
         work = segment_work(spec, w.batch, w.precision, w.optimizer)
-        ms_k = r.timed(warmup + steps, steps, which=k) / steps
-        t_roof = work["gemm_flops"] / (tp * 1e12) + (work["update_bytes"] + work["loss_bytes"]) / (peaks["hbm_gbs"] * 1e9)
-        out["segments"].append({"segment": k, "widths": spec.widths, "ms_per_step": ms_k,
-                                "samples_per_s": w.batch / (ms_k * 1e-3),
-                                "roofline_ms": t_roof * 1e3, "roofline_frac": t_roof * 1e3 / ms_k,
-                                "gemm_tflops": work["gemm_flops"] / (ms_k * 1e-3) / 1e12,
-                                "mem_bytes_peak": seg.mem_bytes()[1]})
+        for key in whole:
+            whole[key] += work[key]
+        ms_k = float(np.median([r.timed(pos + i * steps, steps, which=k) for i in range(3)])) / steps
+        pos += 3 * steps
+        e = {"segment": k, "widths": spec.widths, "ms_per_step": ms_k, "samples_per_s": w.batch / (ms_k * 1e-3),
+             "mem_bytes_peak": seg.mem_bytes()[1]}
+        e.update(step_fractions(work, ms_k, w.precision, peaks))
+        out["segments"].append(e)
+    out["step"] = step_fractions(whole, out["ms_per_step"], w.precision, peaks)
+    out["step"]["segments_alone_ms_sum"] = sum(s_["ms_per_step"] for s_ in out["segments"])
+    out["kernels"], out["roofline"] = kernel_breakdown(r, max(3, min(steps, 20)), pos, peaks)
     if full:
-        # per-kernel device time: the same steps again with events around every launch
-        for seg in r.segs:
-            seg.profile(True)
-        r.run_steps(warmup, steps)
-        torch.cuda.synchronize()
-        kinds = {}
-        for spec, seg in zip(w.segments, r.segs):
-            work = segment_work(spec, w.batch, w.precision, w.optimizer)
-            for name, (n, tot) in seg.profile_read().items():
-                k = kinds.setdefault(name, {"launches": 0, "ms": 0.0, "flops": 0.0, "bytes": 0.0})
-                k["launches"] += n
-                k["ms"] += tot
-                if name in ("fwd_gemm", "dgrad_gemm", "wgrad_gemm"):
-                    k["flops"] += work[name] * steps
-                elif name == "update":          # the update launch also reads dZ for the bias gradient
-                    k["bytes"] += (work["update_bytes"] + work["bias_grad_bytes"]) * steps
-                elif name == "loss":
-                    k["bytes"] += work["loss_bytes"] * steps
-            seg.profile(False)
-        out["kernels"] = {n: {"launches": v["launches"], "ms_total": round(v["ms"], 4),
-                              "avg_us": round(1e3 * v["ms"] / max(v["launches"], 1), 3)} for n, v in kinds.items()}
-        dom = max(kinds, key=lambda n: kinds[n]["ms"])
-        v = kinds[dom]
-        if v["flops"] > 0:
-            achieved = v["flops"] / (v["ms"] * 1e-3) / 1e12
-            out["roofline"] = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": tp, "unit": "TFLOP/s",
-                               "frac": achieved / tp, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
-                               "peak_source": f"{peaks['source']}: sustained bf16 {peaks['bf16_tflops_sustained']} TF/s"
-                                              + (" x 0.5 nominal TF32 ratio" if w.precision == "tf32" else ""),
-                               "timing": "CUDA events around every launch of this kind, same steps re-run after the timed region",
-                               "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
-        else:
-            achieved = v["bytes"] / (v["ms"] * 1e-3) / 1e9
-            out["roofline"] = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                               "peak_source": f"{peaks['source']}: copy bandwidth",
-                               "timing": "CUDA events around every launch of this kind, same steps re-run after the timed region",
-                               "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
         # end to end through the host-buffer entry points: every step reads its batch from pinned host memory
         # (host -> device inside the step) and writes its loss to pinned host memory (device -> host).
         # Timed twice: seg_train_step_host_async (steps enqueued back to back, one synchronisation at the end:
-        # how a training loop calls it) and seg_train_step_host (waits for every loss).
+        # how a training loop calls it) and seg_train_step_host (waits for every loss).  A segment fed label rows
+        # by class takes only the class indices from the host (a pinned -> device copy on its stream).
         e_steps = max(3, min(steps, 50))
-        h2d = sum(w.batch * (spec.widths[0] * (2 if w.precision == "bf16" else 4) + 4) for spec in w.segments)
+        es = 2 if w.precision == "bf16" else 4
+        h2d = sum(w.batch * ((spec.widths[0] * es if r.sil_in[k] is None else 0) + 4) for k, spec in enumerate(w.segments))
         loss_pin = torch.zeros(e_steps + 3, len(r.segs), dtype=torch.float32).pin_memory()
+        cls_dev = [torch.empty(w.batch, dtype=torch.int32, device="cuda") for _ in r.segs]
+        d2h = 0
 
         def e2e_loop(sync_every_step):
+            nonlocal d2h
+            d2h = 0
             for s in range(3 + e_steps):
                 if s == 3:
                     torch.cuda.synchronize()
                     t0 = time.perf_counter()
                 sl = r.batch_slice(s)
                 for k, seg in enumerate(r.segs):
-                    if sync_every_step:
+                    if r.sil_in[k] is not None:
+                        with torch.cuda.stream(r.streams[k]):
+                            cls_dev[k].copy_(r.host_cls[sl], non_blocking=True)
+                            seg.train_step_label_input(r.sil_in[k], cls_dev[k], r.loss[k])
+                            loss_pin[s, k:k + 1].copy_(r.loss[k], non_blocking=True)
+                        if sync_every_step:
+                            r.streams[k].synchronize()
+                    elif sync_every_step:
                         seg.train_step_host(r.host_x[k][sl], r.host_cls[sl])
                     else:
                         seg.train_step_host_async(r.host_x[k][sl], r.host_cls[sl], loss_pin[s, k:k + 1])
+                    d2h += 4
             torch.cuda.synchronize()
             return time.perf_counter() - t0
 
@@ -390,10 +536,13 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
         assert bool(torch.isfinite(loss_pin[3:]).all()) and float(loss_pin[3:].abs().sum()) > 0.0
         out["e2e"] = {"value": e_steps * w.batch / dt_async, "unit": "samples/s", "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": 4 * len(w.segments), "steps": e_steps,
-                      "call": "seg_train_step_host_async per segment and step, one synchronisation after the last step",
+                      "call": "seg_train_step_host_async per segment and step (pinned batch in, loss written to pinned "
+                              "memory), one synchronisation after the last step"
+                              + ("; the label-fed segment: pinned class indices copied in, seg_train_step_label_input, "
+                                 "loss copied out" if any(s_ is not None for s_ in r.sil_in) else ""),
                       "waiting_for_every_loss": {"value": e_steps * w.batch / dt_sync, "unit": "samples/s",
                                                  "call": "seg_train_step_host"}}
-    if full and not w.concurrent:
+    if extras and not w.concurrent:
         # the whole procedure of Section 2, one epoch per segment: train segment k over the resident set in
         # stored order (last partial batch included), store its response, hand it to segment k+1
         from paper_2403_11204_b200 import binding
@@ -409,7 +558,7 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
                                     "stored for the next (seg_train_epochs + seg_forward_dataset)",
                             "samples": n_all, "ms": ms_proc,
                             "samples_per_s": n_all / (ms_proc * 1e-3)}
-    if full and not w.concurrent and len(w.segments) == 2:
+    if extras and not w.concurrent and len(w.segments) == 2:
         # recovery phase of Section 5: the left segment trained through the frozen right one, per step
         from paper_2403_11204_b200 import binding
         rec_loss = torch.zeros(1, device="cuda")
@@ -440,9 +589,8 @@ def measure(workload, steps, warmup, peaks, device_index=0, full=True, n_samples
                              "ratio": e2e_net["mem_bytes_peak"] / seg_peak,
                              "unpartitioned_ms_per_step": e2e_net["ms_per_step"],
                              "segments_ms_per_step_sum": sum(s_["ms_per_step"] for s_ in out["segments"]),
-                             "note": "bytes held by the library per handle (parameters, gradients, optimizer state, "
-                                     "operand copy, activations, dZ, staging); segments trained one at a time need only "
-                                     "the largest segment resident"}
+                             "note": "bytes held by the library per handle; segments trained one at a time need only the "
+                                     "largest segment resident"}
         except Exception as exc:
             out["memory"] = {"error": repr(exc)[:200]}
     return out
@@ -460,14 +608,19 @@ def aggregate_over_ranks(ms_total, steps, batch, world, device="cuda"):
     return world * steps * batch / (ms_total * 1e-3), ms_total
 
 
+def short_segments(segs):
+    keys = ("segment", "ms_per_step", "samples_per_s", "roofline_frac", "tensor_only_frac", "gemm_tflops")
+    return [{k: (round(s[k], 5) if isinstance(s[k], float) else s[k]) for k in keys} for s in segs]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="paper_shaped", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="gemm_large", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--others", default="bf16_wide,gemm_large,multi_cut,tiny,paper_net",
+    ap.add_argument("--others", default="multi_cut,bf16_wide,paper_shaped,tiny,paper_net",
                     help="further workloads summarised in the same line ('' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--samples", type=int, default=0, help="size of the resident data set (0: the workload's own)")
@@ -480,16 +633,21 @@ def main():
     config = {"workload": f"{w.name}: " + " | ".join("-".join(map(str, s.widths)) for s in w.segments),
               "batch": w.batch, "optimizer": w.optimizer, "lr": w.lr, "n_classes": w.n_classes,
               "n_samples": w.n_samples, "label_dist": w.label_dist, "segments_per_step": len(w.segments),
-              "cache": "inputs larger than L2: every step reads the next batch of a resident data set",
+              "segments_in_flight": "concurrently on two streams; segment 1 takes the label rows of the first cut by class "
+                                    "(fully separate variant)" if w.concurrent else "one after another on one stream",
+              "cache": ("inputs larger than L2: every step reads the next batch of a resident data set and streams "
+                        "all weights and optimizer state") if w.n_samples * w.n_features * 2 > L2_BYTES else
+                       "the workload's whole data set is smaller than L2 (no flush: that is its steady state)",
               "parallelism": "replicas only" if world > 1 else "single GPU"}
 
     if args.impl == "reference":
         if rank != 0:
             return
-        base, _ = oracle_samples_per_s(w, budget_s=20.0, max_steps=max(args.steps, 1))
+        base, _ = oracle_samples_per_s(w, budget_s=1e9, max_steps=max(args.steps, 1), warmup=min(args.warmup, 1))
+        rows = min(w.batch, CPU_SAMPLE_BATCH.get(w.name, w.batch))
         line = {"impl": "reference", "metric": "segment train-step samples/sec", "value": base["value"],
                 "unit": "samples/s", "n_gpus": 0, "steps": args.steps, "warmup": args.warmup,
-                "ms_per_step": 1e3 * w.batch / base["value"], "higher_is_better": True, "scaling": "weak",
+                "ms_per_step": 1e3 * rows / base["value"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
                 "cpu_baseline": base,
                 "e2e": {"value": base["value"], "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -506,8 +664,9 @@ def main():
     if world > 1:
         dist.barrier()
     peaks = load_peaks()
+    torch.cuda.set_device(local_rank)
     res = measure(w, args.steps, args.warmup, peaks, device_index=local_rank, full=True,
-                  n_samples=args.samples or None)
+                  n_samples=args.samples or None, extras=not w.concurrent)
     ms_total = res["ms_per_step"] * args.steps
     value, ms_total = aggregate_over_ranks(ms_total, args.steps, w.batch, world)
     if world > 1:
@@ -524,25 +683,43 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16"}[w.precision], "data": "synthetic",
             "config": config, "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"],
-            "roofline": res.get("roofline"), "kernels": res.get("kernels"), "segments": res["segments"],
-            "label_gen_ms": res["label_gen_ms"], "memory": res.get("memory"), "procedure": res.get("procedure"),
-            "recovery": res.get("recovery"), "peaks": peaks}
+            "roofline": res.get("roofline"), "step": res["step"], "repeats": res["repeats"]}
     if not args.no_cpu_baseline:
         line["cpu_baseline"], _ = oracle_samples_per_s(w, budget_s=15.0)
+    line["kernels"] = res.get("kernels")
+    line["segments"] = short_segments(res["segments"])
+    line["product_launches"] = res["product_launches"]
     others = {}
     for name in [n for n in args.others.split(",") if n and n != args.workload]:
         ow = wl.WORKLOADS[name]
         k = max(5, min(args.steps, 30))
         try:
-            r = measure(ow, k, 3, peaks, device_index=local_rank, full=False)
-            others[name] = {"samples_per_s": r["samples_per_s"], "ms_per_step": r["ms_per_step"], "steps": k,
-                            "precision": ow.precision, "optimizer": ow.optimizer, "batch": ow.batch,
-                            "concurrent_streams": ow.concurrent, "memory": r.get("memory"),
-                            "segments": [{kk: s[kk] for kk in ("segment", "ms_per_step", "samples_per_s", "roofline_frac",
-                                                               "gemm_tflops", "mem_bytes_peak")} for s in r["segments"]]}
+            r = measure(ow, k, 3, peaks, device_index=local_rank, full=False, extras=(name == "paper_shaped"))
+            o = {"ms_per_step": round(r["ms_per_step"], 5), "samples_per_s": round(r["samples_per_s"], 1),
+                 "precision": ow.precision, "batch": ow.batch, "step": {kk: round(v, 4) for kk, v in r["step"].items()},
+                 "segments": short_segments(r["segments"]),
+                 "roofline": {kk: r["roofline"][kk] for kk in ("kernel", "bound", "achieved", "peak", "unit", "frac")},
+                 "kernels": {kk: {"share": v["share"], "avg_us": v["avg_us"], "frac_of_peak": v.get("frac_of_peak")}
+                             for kk, v in r["kernels"].items()},
+                 "product_launches": r["product_launches"]}
+            if "memory" in r and "ratio" in r["memory"]:
+                o["memory"] = {kk: r["memory"][kk] for kk in ("largest_segment_bytes", "unpartitioned_bytes", "ratio",
+                                                              "unpartitioned_ms_per_step")}
+            for extra in ("procedure", "recovery"):
+                if extra in r:
+                    o[extra] = {kk: v for kk, v in r[extra].items() if kk != "what"}
+            if ow.n_samples * ow.n_features * 4 < L2_BYTES:
+                o["cache"] = "the workload's whole data set is smaller than L2"
+            others[name] = o
         except Exception as exc:                       # a secondary workload must not cost the headline
             others[name] = {"error": repr(exc)[:200]}
     line["others"] = others
+    line["memory"] = res.get("memory")
+    line["label_gen_ms"] = res["label_gen_ms"]
+    for extra in ("procedure", "recovery"):
+        if extra in res:
+            line[extra] = res[extra]
+    line["peaks"] = peaks
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -20,8 +20,12 @@
  *     nothing.  Device-side problems (a bounded wait that ran out) are recorded in a
  *     status word that seg_poll_status reads.
  *   - Nothing is thrown across this boundary and nothing aborts the process.
- *   - A handle is not thread-safe; different handles may be used from different
- *     threads and on different streams concurrently.
+ *   - A handle is not thread-safe; different handles may be created and used from
+ *     different threads and on different streams concurrently (the library's one-time
+ *     set-up and its per-device caches are synchronised).
+ *   - A handle lives on the device that was current when seg_create ran.  Later calls may
+ *     come with any device current: every call switches to the handle's device for its own
+ *     duration and restores the caller's.
  *
  * Diagnostic environment switches, read when a handle is created (first handle of the
  * process for the kernel-selection ones); all default to off / automatic:
@@ -62,7 +66,8 @@ typedef enum {
   SEG_ERR_CUDA = 5,           /* a CUDA runtime or driver call failed                  */
   SEG_ERR_STATE = 6,          /* call order: e.g. training on labels never generated   */
   SEG_ERR_DEVICE_TIMEOUT = 7, /* a kernel gave up a bounded wait and returned early    */
-  SEG_ERR_NO_DEVICE = 8       /* no CUDA device / not an sm_100 device                 */
+  SEG_ERR_NO_DEVICE = 8,      /* no CUDA device / not an sm_100 device                 */
+  SEG_ERR_CLASS_RANGE = 9     /* a step met a class index outside [0, M) (clamped there) */
 } seg_status;
 
 /* Arithmetic of the matrix products.  Accumulation is always fp32.
@@ -90,7 +95,8 @@ typedef enum { SEG_LABEL_UNIFORM_KAPPA = 0, SEG_LABEL_NORMAL = 1 } seg_label_dis
 typedef enum {
   SEG_GEMM_AUTO = 0,   /* tensor cores for SEG_TF32 / SEG_BF16, FFMA for SEG_FP32 */
   SEG_GEMM_SIMT = 1,   /* FFMA kernels for every precision (same rounding points)  */
-  SEG_GEMM_TCGEN05 = 2 /* tensor-core kernels; SEG_ERR_UNSUPPORTED with SEG_FP32   */
+  SEG_GEMM_TCGEN05 = 2 /* tensor-core kernels only: SEG_ERR_UNSUPPORTED with SEG_FP32, and from any call
+                          whose product the tensor-core path cannot take (no FFMA stand-in) */
 } seg_gemm_backend;
 
 typedef struct {
@@ -132,7 +138,9 @@ SEG_API seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, fl
  * target of each sample's class - or against the class label on the final segment -,
  * backprop inside the segment, optimizer update).
  *   x        [batch][widths[0]]  float (FP32/TF32) or bf16 (BF16)
- *   cls      [batch] int32 class index in [0, M)
+ *   cls      [batch] int32 class index in [0, M).  An index outside that range is clamped to
+ *            it by the step's staging kernel (nothing is read out of bounds) and recorded:
+ *            the next seg_poll_status returns SEG_ERR_CLASS_RANGE.
  *   batch    1..max_batch
  *   loss_out device float, receives the batch loss before the update; may be NULL
  *   y_out    optional [batch][widths[n_layers]] copy of this step's forward output
@@ -236,9 +244,37 @@ SEG_API seg_status seg_mem_bytes(const seg_handle* h, uint64_t* current, uint64_
 /* Number of kernels the handle has launched so far (host counter). */
 SEG_API seg_status seg_launch_count(const seg_handle* h, uint64_t* launches);
 
+/* Matrix-product launches of this handle so far, by kernel family (host counters; counts[4], host):
+ *   [0] tensor-core, one CTA per tile      [1] tensor-core, K split over a cluster
+ *   [2] tensor-core, CTA pair per tile     [3] FFMA
+ * Tests use it to show which kernels actually ran.                                           */
+SEG_API seg_status seg_product_launches(const seg_handle* h, uint64_t* counts);
+
 /* Synchronises the handle's stream and returns SEG_ERR_DEVICE_TIMEOUT if any kernel of
- * this handle gave up a bounded wait since the last poll, SEG_ERR_CUDA on a CUDA error.  */
+ * this handle gave up a bounded wait since the last poll, SEG_ERR_CLASS_RANGE if a step met
+ * a class index outside [0, M), SEG_ERR_CUDA on a CUDA error.  The record is cleared.       */
 SEG_API seg_status seg_poll_status(seg_handle* h);
+
+/* Self-test of the bounded wait every product kernel uses: launches one small block that waits,
+ * with the product kernels' own wait routine, on a barrier nothing ever arrives at, for at most
+ * limit_ns nanoseconds (1,000 .. 1,000,000,000; SEG_ERR_INVALID_ARG otherwise).  The wait runs
+ * out, the block records it in the handle's status word and returns; the next seg_poll_status
+ * reports SEG_ERR_DEVICE_TIMEOUT and the handle stays usable.  Nothing faults or hangs.        */
+SEG_API seg_status seg_selftest_bounded_wait(seg_handle* h, uint64_t limit_ns);
+
+/* Hand-off between segments that live on different devices (Section 2.1: each partition trains on
+ * its own GPU and the only transfer is the previous partition's stored response, once).  Copies
+ * `bytes` bytes from src, device memory on the producer's device (typically the y of
+ * seg_forward_dataset), into dst, device memory on the consumer's device, as one peer copy
+ * enqueued on the producer's stream; the consumer's stream then waits for it, so that a following
+ * seg_train_epochs(consumer, dst, ...) reads the data from its own GPU's memory.  No kernel of
+ * either handle ever reads the other device's memory.  Both handles on one device: an ordinary
+ * device-to-device copy.                                                                         */
+SEG_API seg_status seg_handoff_copy(seg_handle* producer, const void* src, seg_handle* consumer,
+                                    void* dst, uint64_t bytes);
+
+/* Index of the device the handle lives on (host int out). */
+SEG_API seg_status seg_device(const seg_handle* h, int32_t* device);
 
 /* Timing hooks: seg_timer_start / seg_timer_stop record CUDA events on the handle's
  * stream; seg_timer_elapsed_ms synchronises on the stop event (host float out).          */
@@ -268,7 +304,8 @@ SEG_API seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count,
  * - without a handle and without calling cudaMalloc, cudaFree or any allocating routine.
  * The reduction scratch is a static device array of 8 KiB inside the library, present on
  * every GPU that loads the library until the process exits.
- *   out [batch][n_p] float, cls [batch] int32 in [0, n_classes), sil [n_classes][n_p] float,
+ *   out [batch][n_p] float, cls [batch] int32 in [0, n_classes) (an index outside that range is
+ *   clamped to it; nothing is read out of bounds), sil [n_classes][n_p] float,
  *   dz [batch][n_p] float (written), loss_out device float (written; may be NULL),
  *   stream: cudaStream_t.  All device pointers, dense row-major, caller-owned.
  * Limits: n_p <= SEG_NOALLOC_MAX_WIDTH, batch <= SEG_NOALLOC_MAX_BATCH; anything larger

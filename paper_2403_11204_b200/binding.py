@@ -22,6 +22,8 @@ LABEL_DISTS = {"uniform_kappa": SEG_LABEL_UNIFORM_KAPPA, "normal": SEG_LABEL_NOR
 BACKENDS = {"auto": SEG_GEMM_AUTO, "simt": SEG_GEMM_SIMT, "tcgen05": SEG_GEMM_TCGEN05}
 # kind numbers of seg_profile_get (4 is unused: the update launch forms the bias gradient)
 KERNEL_KINDS = {0: "fwd_gemm", 1: "dgrad_gemm", 2: "wgrad_gemm", 3: "loss", 5: "update", 6: "copy"}
+# order of the counters seg_product_launches returns
+PRODUCT_FAMILIES = ("tc_single", "tc_splitk", "tc_pair", "ffma")
 
 
 class seg_config(Structure):
@@ -57,7 +59,11 @@ EXPORTS = {
     "seg_get_activation": (c_int32, [c_void_p, c_int32, c_void_p]),
     "seg_mem_bytes": (c_int32, [c_void_p, POINTER(c_uint64), POINTER(c_uint64)]),
     "seg_launch_count": (c_int32, [c_void_p, POINTER(c_uint64)]),
+    "seg_product_launches": (c_int32, [c_void_p, POINTER(c_uint64)]),
     "seg_poll_status": (c_int32, [c_void_p]),
+    "seg_selftest_bounded_wait": (c_int32, [c_void_p, c_uint64]),
+    "seg_handoff_copy": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64]),
+    "seg_device": (c_int32, [c_void_p, POINTER(c_int32)]),
     "seg_timer_start": (c_int32, [c_void_p]),
     "seg_timer_stop": (c_int32, [c_void_p]),
     "seg_timer_elapsed_ms": (c_int32, [c_void_p, POINTER(c_float)]),
@@ -117,23 +123,46 @@ def label_loss_noalloc(out, cls, sil, relu_mask, dz, loss_out, stream=None):
         raise SegError(status, "seg_label_loss_noalloc")
 
 
+def handoff_copy(producer, src, consumer, dst):
+    """seg_handoff_copy: the stored response `src` (on the producer's device) into `dst` (same shape and
+    dtype, on the consumer's device); the consumer's stream waits for the copy."""
+    assert src.is_cuda and dst.is_cuda and src.is_contiguous() and dst.is_contiguous()
+    assert src.shape == dst.shape and src.dtype == dst.dtype
+    producer._check(producer.lib.seg_handoff_copy(producer.h, _ptr(src), consumer.h, _ptr(dst),
+                                                  src.numel() * src.element_size()), "seg_handoff_copy")
+
+
 def train_partitioned(segments, x, cls, batch, epochs):
     """The paper's training procedure (Section 2, two or more partitions): segment k is trained for
     epochs[k] passes on the stored response of segment k-1 (segment 0 on x) against its own
     intermediate labels - the last segment against the class labels - and only then is its response
     over the whole set computed and handed to segment k+1.  Returns the per-step losses of every
     segment (device tensors) and the last segment's input.  Marshalling only: every step runs in
-    seg_train_epochs / seg_forward_dataset."""
+    seg_train_epochs / seg_forward_dataset.
+
+    Segments may live on different devices (Section 2.1: one partition per GPU, the only transfer being
+    the previous partition's stored response, once): x and cls are on the first segment's device; the
+    response of segment k is copied into the next segment's device by seg_handoff_copy, the class
+    indices by torch, before that segment's first step."""
     import torch
     losses = []
-    cur = x
+    cur, cur_cls = x, cls
     for k, (seg, n_ep) in enumerate(zip(segments, epochs)):
         steps = n_ep * (-(-cur.shape[0] // batch))
-        l = torch.zeros(max(steps, 1), device="cuda")
-        seg.train_epochs(cur, cls, batch, n_ep, l)
+        with torch.cuda.device(seg.device):
+            l = torch.zeros(max(steps, 1), device="cuda")
+        seg.train_epochs(cur, cur_cls, batch, n_ep, l)
         losses.append(l[:steps])
         if k + 1 < len(segments):
-            cur = seg.forward_dataset(cur, batch)
+            nxt = segments[k + 1]
+            resp = seg.forward_dataset(cur, batch)
+            if nxt.device != seg.device:
+                dst = nxt._empty(*resp.shape, dtype=resp.dtype)
+                handoff_copy(seg, resp, nxt, dst)
+                seg.stream.synchronize()             # resp may be released once the copy has run
+                resp = dst
+                cur_cls = cur_cls.to(f"cuda:{nxt.device}")
+            cur = resp
     return losses, cur
 
 
@@ -160,17 +189,18 @@ class Segment:
 
     def __init__(self, widths, n_classes, is_final, *, precision="fp32", optimizer="sgd", lr=0.01,
                  momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, max_batch=256, segment_id=0,
-                 init_seed=2, last_relu=None, gemm_backend="auto", stream=None):
+                 init_seed=2, last_relu=None, gemm_backend="auto", stream=None, device=None):
         import torch
         self._torch = torch
         if not torch.cuda.is_available():
             raise RuntimeError("Segment needs a CUDA device; there is no CPU path")
         self.lib = load()
+        self.device = torch.cuda.current_device() if device is None else int(device)
         self.widths = [int(w) for w in widths]
         self.n_layers = len(self.widths) - 1
         self.n_classes, self.is_final, self.precision = int(n_classes), bool(is_final), precision
         self.max_batch = int(max_batch)
-        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         self._warr = (c_int32 * len(self.widths))(*self.widths)
         cfg = seg_config(self.n_layers, self._warr, self.n_classes, int(self.is_final),
                          -1 if last_relu is None else int(bool(last_relu)), int(segment_id),
@@ -178,7 +208,8 @@ class Segment:
                          self.max_batch, BACKENDS[gemm_backend], int(init_seed),
                          c_void_p(self.stream.cuda_stream))
         self.h = c_void_p()
-        self._check(self.lib.seg_create(byref(cfg), byref(self.h)), "seg_create")
+        with torch.cuda.device(self.device):          # the handle lives on the device current at seg_create
+            self._check(self.lib.seg_create(byref(cfg), byref(self.h)), "seg_create")
         self.act_dtype = torch.bfloat16 if precision == "bf16" else torch.float32
         self.out_dtype = torch.float32 if self.is_final else self.act_dtype
         self.last_batch = 0
@@ -193,7 +224,7 @@ class Segment:
             raise SegError(status, detail)
 
     def _empty(self, *shape, dtype=None):
-        with self._torch.cuda.stream(self.stream):
+        with self._torch.cuda.device(self.device), self._torch.cuda.stream(self.stream):
             return self._torch.empty(*shape, dtype=dtype or self._torch.float32, device="cuda")
 
     def close(self):
@@ -338,8 +369,17 @@ class Segment:
         self._check(self.lib.seg_launch_count(self.h, byref(n)), "seg_launch_count")
         return n.value
 
+    def product_launches(self):
+        """seg_product_launches as a dict: launches per product-kernel family."""
+        c = (c_uint64 * 4)()
+        self._check(self.lib.seg_product_launches(self.h, c), "seg_product_launches")
+        return dict(zip(PRODUCT_FAMILIES, (int(v) for v in c)))
+
     def poll(self):
         self._check(self.lib.seg_poll_status(self.h), "seg_poll_status")
+
+    def selftest_bounded_wait(self, limit_ns):
+        self._check(self.lib.seg_selftest_bounded_wait(self.h, int(limit_ns)), "seg_selftest_bounded_wait")
 
     def timer_start(self):
         self._check(self.lib.seg_timer_start(self.h))

@@ -20,8 +20,12 @@ enum Epilogue : int {
   EPI_PLAIN = 2      // wgrad:   store the fp32 product
 };
 
-// Device status word values (written by kernels that give up a bounded wait).
-enum DevStatus : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
+// Device status word: bits OR-ed in by kernels (a bounded wait that ran out; a class index outside
+// [0, M) met and clamped by the input staging).
+enum DevStatus : int { DEV_OK = 0, DEV_TIMEOUT = 1, DEV_BAD_CLASS = 2 };
+
+// Families of matrix-product kernels (reported per handle by seg_product_launches).
+enum Family : int { FAM_TC_SINGLE = 0, FAM_TC_SPLITK = 1, FAM_TC_PAIR = 2, FAM_SIMT = 3, FAM_COUNT = 4 };
 
 // The loss of a non-final segment fused into the epilogue of its last forward product when the
 // split-K kernel runs it (Section 2: the target is the intermediate label of the sample's class; the
@@ -75,8 +79,11 @@ constexpr int kSimtTileFloats = 64 * 64;
 cudaError_t launch_gemm_simt(const GemmDesc& g, cudaStream_t s);
 int gemm_simt_slots(int M, int N, int K);   // workspace slots (partial 64 x 64 tiles) a split of this product would use
 // Tensor-core path.  Returns cudaErrorNotSupported when the shape/stride does not fit its TMA rules.
-cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s);
-bool gemm_tc_init();   // resolves the driver entry point needed for tensor maps
+// *family (may be null) receives the Family of the kernel that was launched.
+cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s, int* family = nullptr);
+bool gemm_tc_init();   // resolves the driver entry point needed for tensor maps (once per process, thread-safe)
+// One block that waits, with the product kernels' bounded wait, on a barrier nothing arrives at.
+cudaError_t launch_wait_selftest(int* dev_status, uint64_t limit_ns, cudaStream_t s);
 // True when launch_gemm_tc would take the intermediate-label loss into the forward product M x N x K.
 bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32);
 
@@ -88,7 +95,7 @@ cudaError_t launch_init_uniform(float* dst, int rows, int cols, int64_t ld, uint
 // loss kernels: write dZ (dz_dt, rounded by dz_round) and a deterministic batch loss, which goes to
 // the address stored in the device slot *loss_dst (the input-staging launch of the step fills it)
 cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const int32_t* cls,
-                            const float* sil, int n_p, int batch, int relu_mask,
+                            const float* sil, int n_classes, int n_p, int batch, int relu_mask,
                             void* dz, int dz_dt, int dz_round, int64_t ld_dz,
                             float* partials, unsigned int* counter, float* const* loss_dst, cudaStream_t s);
 cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const int32_t* cls,
@@ -122,15 +129,17 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s);
 
 // copies with pitch / dtype / rounding conversion: dst[r][c] = cvt(src[r][c])
 cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt,
-                          int64_t ld_src, int rows, int cols, int round, cudaStream_t s);
+                          int64_t ld_src, int64_t rows, int64_t cols, int round, cudaStream_t s);
 // the same copy plus an int32 vector copy (class indices) in one launch; when t is not null the
 // launch also advances the step counter: t += 1, bc = {1 - beta1^t, 1 - beta2^t}; when gather_src is not
 // null, row r of the destination is row cls[r] of that fp32 [classes][cols] matrix instead of src's row r;
-// when loss_dst is not null the launch stores loss_out there (the step's loss kernel reads it back)
+// when loss_dst is not null the launch stores loss_out there (the step's loss kernel reads it back).
+// Class indices are clamped to [0, n_classes) on the way; one outside sets DEV_BAD_CLASS in *dev_status.
 cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2,
-                                const float* gather_src, float* loss_out, float** loss_dst, cudaStream_t s);
+                                const float* gather_src, float* loss_out, float** loss_dst,
+                                int n_classes, int* dev_status, cudaStream_t s);
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // Kernels of one stream are launched with programmatic stream serialisation: a kernel may become

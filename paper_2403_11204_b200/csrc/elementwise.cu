@@ -68,35 +68,78 @@ __device__ void finish_loss(float block_total, float* partials, unsigned int* co
 
 // Non-final segment: target of sample b is row cls[b] of the label matrix (gathered here, never
 // materialised per sample);  loss = mean (a - t)^2,  dZ = 2 (a - t) / (B N_P) * [a > 0].
-template <typename TOut, typename TDz>
+// A thread handles VEC consecutive columns of one row per pass (VEC = 8: 16-byte accesses for bf16,
+// two for fp32 and for the fp32 targets); VEC = 1 serves widths that are not multiples of 8.  A class
+// index outside [0, n_classes) is clamped, so that nothing is read out of bounds.
+template <typename TOut, typename TDz, int VEC>
 __global__ void __launch_bounds__(kLossThreads)
 mse_loss_kernel(const TOut* __restrict__ out, int64_t ld_out, const int32_t* __restrict__ cls,
-                const float* __restrict__ sil, int n_p, int batch, int relu_mask,
+                const float* __restrict__ sil, int n_classes, int n_p, int batch, int relu_mask,
                 TDz* __restrict__ dz, int dz_round, int64_t ld_dz, float* partials,
                 unsigned int* counter, float* loss_out, float* const* loss_dst) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[32];
-  const int64_t total = (int64_t)batch * n_p;
-  const float gscale = 2.0f / (float)total;
+  const float gscale = 2.0f / (float)((int64_t)batch * n_p);
   float acc = 0.f;
-  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
-       e += (int64_t)gridDim.x * blockDim.x) {
-    const int b = (int)(e / n_p), i = (int)(e % n_p);
-    float a;
-    if constexpr (sizeof(TOut) == 2) a = __bfloat162float(out[b * ld_out + i]);
-    else a = out[b * ld_out + i];
-    const float t = __ldg(sil + (int64_t)__ldg(cls + b) * n_p + i);
-    const float d = a - t;
-    acc = fmaf(d, d, acc);
-    float g = d * gscale;
-    if (relu_mask && !(a > 0.f)) g = 0.f;
-    g = apply_round(g, dz_round);
-    if constexpr (sizeof(TDz) == 2) dz[b * ld_dz + i] = __float2bfloat16_rn(g);
-    else dz[b * ld_dz + i] = g;
+  const unsigned int groups_per_row = (unsigned int)(n_p / VEC);
+  const int64_t n_groups = (int64_t)batch * groups_per_row;
+  for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < n_groups;
+       v += (int64_t)gridDim.x * blockDim.x) {
+    const int b = (int)(v / groups_per_row);
+    const int i = (int)(v - (int64_t)b * groups_per_row) * VEC;
+    const int c = min(max(__ldg(cls + b), 0), n_classes - 1);
+    const float* trow = sil + (int64_t)c * n_p + i;
+    float a[VEC], t[VEC], g[VEC];
+    if constexpr (VEC == 8) {
+      if constexpr (sizeof(TOut) == 2) {
+        const uint4 q = *reinterpret_cast<const uint4*>(out + (int64_t)b * ld_out + i);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          a[2 * j] = __uint_as_float(w[j] << 16);
+          a[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+        }
+      } else {
+        const float4 q0 = *reinterpret_cast<const float4*>(out + (int64_t)b * ld_out + i);
+        const float4 q1 = *reinterpret_cast<const float4*>(out + (int64_t)b * ld_out + i + 4);
+        a[0] = q0.x; a[1] = q0.y; a[2] = q0.z; a[3] = q0.w; a[4] = q1.x; a[5] = q1.y; a[6] = q1.z; a[7] = q1.w;
+      }
+      const float4 t0 = __ldg(reinterpret_cast<const float4*>(trow));
+      const float4 t1 = __ldg(reinterpret_cast<const float4*>(trow + 4));
+      t[0] = t0.x; t[1] = t0.y; t[2] = t0.z; t[3] = t0.w; t[4] = t1.x; t[5] = t1.y; t[6] = t1.z; t[7] = t1.w;
+    } else {
+      if constexpr (sizeof(TOut) == 2) a[0] = __bfloat162float(out[(int64_t)b * ld_out + i]);
+      else a[0] = out[(int64_t)b * ld_out + i];
+      t[0] = __ldg(trow);
+    }
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const float d = a[j] - t[j];
+      acc = fmaf(d, d, acc);
+      float gj = d * gscale;
+      if (relu_mask && !(a[j] > 0.f)) gj = 0.f;
+      g[j] = apply_round(gj, dz_round);
+    }
+    if constexpr (VEC == 8) {
+      if constexpr (sizeof(TDz) == 2) {
+        uint4 q;
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(g[0], g[1]), p1 = __floats2bfloat162_rn(g[2], g[3]);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(g[4], g[5]), p3 = __floats2bfloat162_rn(g[6], g[7]);
+        q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
+        q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
+        *reinterpret_cast<uint4*>(dz + (int64_t)b * ld_dz + i) = q;
+      } else {
+        *reinterpret_cast<float4*>(dz + (int64_t)b * ld_dz + i) = make_float4(g[0], g[1], g[2], g[3]);
+        *reinterpret_cast<float4*>(dz + (int64_t)b * ld_dz + i + 4) = make_float4(g[4], g[5], g[6], g[7]);
+      }
+    } else {
+      if constexpr (sizeof(TDz) == 2) dz[(int64_t)b * ld_dz + i] = __float2bfloat16_rn(g[0]);
+      else dz[(int64_t)b * ld_dz + i] = g[0];
+    }
   }
   const float bt = block_sum(acc, red);
-  finish_loss(bt, partials, counter, loss_out, loss_dst, 1.0f / (float)total, red);
+  finish_loss(bt, partials, counter, loss_out, loss_dst, 1.0f / (float)((int64_t)batch * n_p), red);
 }
 
 // Final segment: one warp per sample;  p = softmax(z) with the row maximum subtracted,
@@ -251,10 +294,10 @@ update_kernel(UpdateArgs u, int bias_blocks, int bias_cols) {
 
 __global__ void __launch_bounds__(256)
 copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt, int64_t ld_src,
-              int rows, int cols, int round) {
+              int64_t rows, int64_t cols, int round) {
   pdl_wait();
   pdl_trigger();
-  const int64_t total = (int64_t)rows * cols;
+  const int64_t total = rows * cols;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
        e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = e / cols, c = e % cols;
@@ -266,11 +309,13 @@ copy2d_kernel(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt
 __global__ void __launch_bounds__(256)
 stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows, int cols,
                     int round, int32_t* cls_dst, const int32_t* cls_src, unsigned long long* t, float* bc,
-                    float beta1, float beta2, const float* gather_src, float* loss_out, float** loss_dst) {
+                    float beta1, float beta2, const float* gather_src, float* loss_out, float** loss_dst,
+                    int n_classes, int* dev_status) {
   pdl_wait();
   pdl_trigger();
   const int64_t total = (int64_t)rows * cols;
   const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const int64_t n_threads = (int64_t)gridDim.x * blockDim.x;
   if (tid == 0 && loss_dst != nullptr) *loss_dst = loss_out;   // where this step's loss kernel writes the loss
   if (tid == 0 && t != nullptr) {           // step counter and Adam bias corrections of this step
     const unsigned long long step = *t + 1ull;
@@ -279,16 +324,42 @@ stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t 
     bc[1] = (float)(1.0 - pow((double)beta2, (double)step));
   }
   const int esz = dt == DT_BF16 ? 2 : 4;
-  const bool wide = gather_src == nullptr && ((cols * esz) & 15) == 0 && ((ld_src * esz) & 15) == 0 &&
-                    ((ld_dst * esz) & 15) == 0 &&
-                    ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0;
-  if (wide) {
+  const bool dst_wide = ((cols * esz) & 15) == 0 && ((ld_dst * esz) & 15) == 0 &&
+                        (reinterpret_cast<uintptr_t>(dst) & 15u) == 0;
+  if (gather_src != nullptr && dst_wide && (cols & 7) == 0) {
+    // the input of sample r is row cls[r] of an fp32 label matrix (the fully separate variant): eight
+    // columns per thread and pass, 16-byte loads of the label row, one or two 16-byte stores
+    const int groups_per_row = cols / 8;
+    const int64_t n_groups = (int64_t)rows * groups_per_row;
+    for (int64_t v = tid; v < n_groups; v += n_threads) {
+      const int r = (int)(v / groups_per_row), c = (int)(v - (int64_t)r * groups_per_row) * 8;
+      const int k = min(max(__ldg(cls_src + r), 0), n_classes - 1);
+      const float4 q0 = __ldg(reinterpret_cast<const float4*>(gather_src + (int64_t)k * cols + c));
+      const float4 q1 = __ldg(reinterpret_cast<const float4*>(gather_src + (int64_t)k * cols + c + 4));
+      float f[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+      if (dt == DT_BF16) {
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(f[0], f[1]), p1 = __floats2bfloat162_rn(f[2], f[3]);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(f[4], f[5]), p3 = __floats2bfloat162_rn(f[6], f[7]);
+        uint4 q;
+        q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
+        q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(dst) + (int64_t)r * ld_dst + c) = q;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = apply_round(f[j], round);
+        float* drow = reinterpret_cast<float*>(dst) + (int64_t)r * ld_dst + c;
+        *reinterpret_cast<float4*>(drow) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4*>(drow + 4) = make_float4(f[4], f[5], f[6], f[7]);
+      }
+    }
+  } else if (gather_src == nullptr && dst_wide && ((ld_src * esz) & 15) == 0 &&
+             (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
     // 16 bytes per access: rows are whole numbers of 16-byte groups on both sides
     const int vec_per_row = cols * esz / 16;
     const int64_t n_vec = (int64_t)rows * vec_per_row;
     const char* sb = reinterpret_cast<const char*>(src);
     char* db = reinterpret_cast<char*>(dst);
-    for (int64_t v = tid; v < n_vec; v += (int64_t)gridDim.x * blockDim.x) {
+    for (int64_t v = tid; v < n_vec; v += n_threads) {
       const int64_t r = v / vec_per_row, c = v % vec_per_row;
       uint4 q = __ldg(reinterpret_cast<const uint4*>(sb + r * ld_src * esz) + c);
       if (round == RND_TF32 && dt == DT_F32) {
@@ -300,15 +371,25 @@ stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t 
       reinterpret_cast<uint4*>(db + r * ld_dst * esz)[c] = q;
     }
   } else {
-    for (int64_t e = tid; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    for (int64_t e = tid; e < total; e += n_threads) {
       const int64_t r = e / cols, c = e % cols;
-      // gather_src: the input of sample r is row cls[r] of an fp32 label matrix (the fully separate variant)
-      const float raw = gather_src ? __ldg(gather_src + (int64_t)__ldg(cls_src + r) * cols + c)
-                                   : load_as_float(src, dt, r * ld_src + c);
+      float raw;
+      if (gather_src) {
+        const int k = min(max(__ldg(cls_src + r), 0), n_classes - 1);
+        raw = __ldg(gather_src + (int64_t)k * cols + c);
+      } else {
+        raw = load_as_float(src, dt, r * ld_src + c);
+      }
       store_from_float(dst, dt, r * ld_dst + c, apply_round(raw, round));
     }
   }
-  for (int64_t i = tid; i < rows; i += (int64_t)gridDim.x * blockDim.x) cls_dst[i] = cls_src[i];
+  // class indices: clamped into [0, n_classes); one outside that range is recorded in the status word
+  for (int64_t i = tid; i < rows; i += n_threads) {
+    const int k = cls_src[i];
+    const int kc = min(max(k, 0), n_classes - 1);
+    if (kc != k && dev_status != nullptr) atomicOr(dev_status, (int)DEV_BAD_CLASS);
+    cls_dst[i] = kc;
+  }
 }
 
 int grid_for(int64_t work_items, int threads, int max_blocks) {
@@ -321,23 +402,30 @@ int grid_for(int64_t work_items, int threads, int max_blocks) {
 
 int loss_max_partials() { return kMaxLossBlocks; }
 
+// Eight columns per thread when every row segment involved is 16-byte aligned, one otherwise.
+bool mse_wide(const void* out, int64_t ld_out, const void* dz, int64_t ld_dz, const float* sil, int n_p) {
+  return (n_p & 7) == 0 && (ld_out & 7) == 0 && (ld_dz & 7) == 0 &&
+         ((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(dz) | reinterpret_cast<uintptr_t>(sil)) & 15u) == 0;
+}
+
 cudaError_t launch_mse_loss(const void* out, int out_dt, int64_t ld_out, const int32_t* cls,
-                            const float* sil, int n_p, int batch, int relu_mask, void* dz,
+                            const float* sil, int n_classes, int n_p, int batch, int relu_mask, void* dz,
                             int dz_dt, int dz_round, int64_t ld_dz, float* partials,
                             unsigned int* counter, float* const* loss_dst, cudaStream_t s) {
   float* const loss_out = nullptr;
-  const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
+  const bool wide = mse_wide(out, ld_out, dz, ld_dz, sil, n_p);
+  const int grid = grid_for((int64_t)batch * n_p, kLossThreads * (wide ? 16 : 4), kMaxLossBlocks);
+#define SEGK_MSE(TO, TD, V)                                                                              \
+  launch_k(mse_loss_kernel<TO, TD, V>, dim3(grid), dim3(kLossThreads), 0, s, (const TO*)out, ld_out, cls, \
+           sil, n_classes, n_p, batch, relu_mask, (TD*)dz, dz_round, ld_dz, partials, counter, loss_out, loss_dst)
   if (out_dt == DT_BF16 && dz_dt == DT_BF16) {
-    launch_k(mse_loss_kernel<__nv_bfloat16, __nv_bfloat16>, dim3(grid), dim3(kLossThreads), 0, s, 
-        (const __nv_bfloat16*)out, ld_out, cls, sil, n_p, batch, relu_mask, (__nv_bfloat16*)dz,
-        dz_round, ld_dz, partials, counter, loss_out, loss_dst);
+    if (wide) SEGK_MSE(__nv_bfloat16, __nv_bfloat16, 8); else SEGK_MSE(__nv_bfloat16, __nv_bfloat16, 1);
   } else if (out_dt == DT_F32 && dz_dt == DT_F32) {
-    launch_k(mse_loss_kernel<float, float>, dim3(grid), dim3(kLossThreads), 0, s, 
-        (const float*)out, ld_out, cls, sil, n_p, batch, relu_mask, (float*)dz, dz_round, ld_dz,
-        partials, counter, loss_out, loss_dst);
+    if (wide) SEGK_MSE(float, float, 8); else SEGK_MSE(float, float, 1);
   } else {
     return cudaErrorInvalidValue;
   }
+#undef SEGK_MSE
   return cudaGetLastError();
 }
 
@@ -383,18 +471,19 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
 cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* src, int64_t ld_src, int rows,
                                 int cols, int round, int32_t* cls_dst, const int32_t* cls_src,
                                 unsigned long long* t, float* bc, float beta1, float beta2,
-                                const float* gather_src, float* loss_out, float** loss_dst, cudaStream_t s) {
+                                const float* gather_src, float* loss_out, float** loss_dst,
+                                int n_classes, int* dev_status, cudaStream_t s) {
   const int esz = dt == DT_BF16 ? 2 : 4;
   const int grid = grid_for((int64_t)rows * cols * esz / 16, 256, 148 * 8);   // one 16-byte group per thread and pass
   launch_k(stage_inputs_kernel, dim3(grid), dim3(256), 0, s, dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
-                                           beta1, beta2, gather_src, loss_out, loss_dst);
+                                           beta1, beta2, gather_src, loss_out, loss_dst, n_classes, dev_status);
   return cudaGetLastError();
 }
 
 cudaError_t launch_copy2d(void* dst, int dst_dt, int64_t ld_dst, const void* src, int src_dt,
-                          int64_t ld_src, int rows, int cols, int round, cudaStream_t s) {
-  if ((int64_t)rows * cols == 0) return cudaSuccess;
-  const int grid = grid_for((int64_t)rows * cols, 256 * 4, 148 * 8);
+                          int64_t ld_src, int64_t rows, int64_t cols, int round, cudaStream_t s) {
+  if (rows <= 0 || cols <= 0) return cudaSuccess;
+  const int grid = grid_for(rows * cols, 256 * 4, 148 * 8);
   launch_k(copy2d_kernel, dim3(grid), dim3(256), 0, s, dst, dst_dt, ld_dst, src, src_dt, ld_src, rows, cols, round);
   return cudaGetLastError();
 }
@@ -453,9 +542,14 @@ extern "C" SEG_API seg_status seg_label_loss_noalloc(const float* out, const int
   unsigned int* counter = reinterpret_cast<unsigned int*>(reinterpret_cast<unsigned char*>(scratch) + 4096);
   // the array keeps whatever the previous call left: the arrival counter must start at zero
   if (cudaMemsetAsync(counter, 0, sizeof(unsigned int), s) != cudaSuccess) { cudaGetLastError(); return SEG_ERR_CUDA; }
-  const int grid = grid_for((int64_t)batch * n_p, kLossThreads * 4, kMaxLossBlocks);
-  mse_loss_kernel<float, float><<<grid, kLossThreads, 0, s>>>(out, n_p, cls, sil, n_p, batch, relu_mask ? 1 : 0, dz,
-                                                             RND_NONE, n_p, partials, counter, loss_out, nullptr);
+  const bool wide = mse_wide(out, n_p, dz, n_p, sil, n_p);
+  const int grid = grid_for((int64_t)batch * n_p, kLossThreads * (wide ? 16 : 4), kMaxLossBlocks);
+  if (wide)
+    mse_loss_kernel<float, float, 8><<<grid, kLossThreads, 0, s>>>(out, n_p, cls, sil, n_classes, n_p, batch, relu_mask ? 1 : 0,
+                                                                  dz, RND_NONE, n_p, partials, counter, loss_out, nullptr);
+  else
+    mse_loss_kernel<float, float, 1><<<grid, kLossThreads, 0, s>>>(out, n_p, cls, sil, n_classes, n_p, batch, relu_mask ? 1 : 0,
+                                                                  dz, RND_NONE, n_p, partials, counter, loss_out, nullptr);
   if (cudaGetLastError() != cudaSuccess) return SEG_ERR_CUDA;
   return SEG_OK;
 }

@@ -39,6 +39,8 @@
 #include <stdlib.h>
 
 #include <algorithm>
+#include <atomic>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -81,8 +83,9 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait.  Returns false when the wait was abandoned (own time-out or another role's abort).
+// The product kernels pass the compile-time limit; the self-test kernel passes a short one.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* dev_status) {
+                                          int* dev_status, uint64_t limit_ns = WAIT_LIMIT_NS) {
   uint32_t spins = 0;
   uint64_t t0 = 0;
   while (!mbar_try_wait(bar, parity)) {
@@ -90,9 +93,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) {
+      else if (now - t0 > limit_ns) {
         *abort_flag = 1;
-        atomicExch(dev_status, (int)DEV_TIMEOUT);
+        atomicOr(dev_status, (int)DEV_TIMEOUT);
         return false;
       }
     }
@@ -1019,14 +1022,34 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
-int g_num_sms = 0;      // every device of one process is assumed to be the same part
+constexpr int kMaxDevices = 64;
 
 int current_device_slot() {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
   return dev;
 }
-bool g_init_done = false, g_init_ok = false;
+// SM count of the current device (cached per device; handles may live on different devices)
+int num_sms() {
+  static std::atomic<int> cache[kMaxDevices];
+  const int slot = current_device_slot();
+  int n = cache[slot].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, slot) != cudaSuccess || n <= 0) { cudaGetLastError(); return 148; }
+  cache[slot].store(n, std::memory_order_relaxed);
+  return n;
+}
+// cudaFuncSetAttribute once per kernel and device (the call itself is idempotent, so a race only repeats it)
+template <typename Kern>
+cudaError_t ensure_dynamic_smem(Kern kern, int bytes, std::atomic<bool>* flags) {
+  std::atomic<bool>& done = flags[current_device_slot()];
+  if (done.load(std::memory_order_acquire)) return cudaSuccess;
+  cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (err == cudaSuccess) done.store(true, std::memory_order_release);
+  return err;
+}
+std::once_flag g_init_once;
+bool g_init_ok = false;
 bool g_allow_splitk = true;
 bool g_allow_pairs = true;
 long g_pair_min_tiles = 0;      // SEG_PAIR_MIN_TILES: CTA pairs exactly from this many 256 x 256 tiles on (0: cost model)
@@ -1053,15 +1076,10 @@ cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const G
                            const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   using L = SmemLayout<BLOCK_N>;
   auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N>;
-  static bool attr_set_dev[64] = {};      // the attribute is per device
-  bool& attr_set = attr_set_dev[current_device_slot()];
-  if (!attr_set) {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
-    if (err != cudaSuccess) return err;
-    attr_set = true;
-  }
+  static std::atomic<bool> attr_set_dev[kMaxDevices];      // the attribute is per device
+  if (cudaError_t err = ensure_dynamic_smem(kern, L::TOTAL, attr_set_dev); err != cudaSuccess) return err;
   const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + BLOCK_N - 1) / BLOCK_N);
-  const int grid = tiles < g_num_sms ? tiles : g_num_sms;
+  const int grid = tiles < num_sms() ? tiles : num_sms();
   return launch_k(kern, dim3(grid), dim3(NUM_THREADS), L::TOTAL, s, ma, mb, g.M, g.N, g.K, e, dev_status);
 }
 
@@ -1079,13 +1097,8 @@ template <bool TF32, bool A_MN, bool B_MN, bool LOSS = false>
 cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                                   const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
   auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN, LOSS>;
-  static bool attr_set_dev[64] = {};      // the attribute is per device
-  bool& attr_set = attr_set_dev[current_device_slot()];
-  if (!attr_set) {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SPLITK_SMEM);
-    if (err != cudaSuccess) return err;
-    attr_set = true;
-  }
+  static std::atomic<bool> attr_set_dev[kMaxDevices];      // the attribute is per device
+  if (cudaError_t err = ensure_dynamic_smem(kern, SPLITK_SMEM, attr_set_dev); err != cudaSuccess) return err;
   const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + SPLITK_BLOCK_N - 1) / SPLITK_BLOCK_N);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
@@ -1122,7 +1135,7 @@ int pick_split(int M, int N, int K, bool tf32) {
   int best = 1;
   double best_us = 0.27 * num_k;
   for (int sp : {2, 4}) {
-    if (tiles * sp > g_num_sms) break;
+    if (tiles * sp > num_sms()) break;
     const double us = 0.27 * ((num_k + sp - 1) / sp) + 2.0;
     if (us < best_us - 0.5) { best = sp; best_us = us; }
   }
@@ -1133,15 +1146,10 @@ template <bool TF32, bool A_MN, bool B_MN>
 cudaError_t launch_pair_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                                 const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   auto kern = gemm_tc_pair_kernel<TF32, A_MN, B_MN>;
-  static bool attr_set_dev[64] = {};      // the attribute is per device
-  bool& attr_set = attr_set_dev[current_device_slot()];
-  if (!attr_set) {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
-    if (err != cudaSuccess) return err;
-    attr_set = true;
-  }
+  static std::atomic<bool> attr_set_dev[kMaxDevices];      // the attribute is per device
+  if (cudaError_t err = ensure_dynamic_smem(kern, PAIR_SMEM, attr_set_dev); err != cudaSuccess) return err;
   const int tiles = ((g.M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((g.N + PAIR_TILE_N - 1) / PAIR_TILE_N);
-  const int pairs = std::min(tiles, g_num_sms / 2);
+  const int pairs = std::min(tiles, num_sms() / 2);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
@@ -1177,25 +1185,25 @@ Choice pick_kernel(int M, int N, int K, bool tf32, bool throughput) {
   for (int bn : {64, 128, 256}) {
     if (bn > 64 && bn / 2 >= N) continue;                  // do not use a tile twice as wide as N
     const long tiles = (long)tiles_m * ((N + bn - 1) / bn);
-    const long rounds = (tiles + g_num_sms - 1) / g_num_sms;
+    const long rounds = (tiles + num_sms() - 1) / num_sms();
     const double per_kb = (16.0 + bn / 8.0) / 120.0;       // KiB per k-block / (KiB per us)
     double us = rounds * (num_k * per_kb + 0.4 + bn / 128.0);   // + per-tile epilogue not hidden
     // beside other kernels the SM time taken counts as well: latency + tiles x time of a tile / SMs, with the
     // measured fixed cost of a tile (wider tiles drain more columns and allocate more tensor memory)
     if (throughput) {
       const double t = num_k * per_kb + 3.5 + bn / 48.0;
-      us = rounds * t + (double)tiles * t / g_num_sms;
+      us = rounds * t + (double)tiles * t / num_sms();
     }
     if (us < best.us) best = Choice{0, bn, us};
   }
   if (g_allow_pairs && M >= 256 && N >= 256 && K >= 256) {
     const long tiles = (long)((M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((N + PAIR_TILE_N - 1) / PAIR_TILE_N);
-    const long pairs = g_num_sms / 2;
+    const long pairs = num_sms() / 2;
     const long rounds = (tiles + pairs - 1) / pairs;
     double us = rounds * (num_k * (32.0 / 120.0) + 0.4 + 2.0);
     if (throughput) {
       const double t = num_k * (32.0 / 120.0) + 9.0;          // measured: a pair's fixed cost is about 9 us
-      us = rounds * t + (double)(2 * tiles) * t / g_num_sms;
+      us = rounds * t + (double)(2 * tiles) * t / num_sms();
     }
     if (g_pair_min_tiles > 0) {                            // diagnostic override: pairs from that many tiles on
       if (tiles >= g_pair_min_tiles) best = Choice{1, PAIR_HALF_N, us};
@@ -1209,27 +1217,45 @@ Choice pick_kernel(int M, int N, int K, bool tf32, bool throughput) {
 }  // namespace
 
 bool gemm_tc_init() {
-  if (g_init_done) return g_init_ok;
-  g_init_done = true;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
-    cudaGetLastError();
-    return false;
-  }
-  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return false;
-  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-  const char* env = getenv("SEG_NO_SPLITK");
-  if (env && env[0] == '1') g_allow_splitk = false;
-  env = getenv("SEG_NO_PAIRS");
-  if (env && env[0] == '1') g_allow_pairs = false;
-  env = getenv("SEG_PAIR_MIN_TILES");
-  if (env) g_pair_min_tiles = atol(env);
-  g_init_ok = g_num_sms > 0;
+  std::call_once(g_init_once, [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+      cudaGetLastError();
+      return;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    const char* env = getenv("SEG_NO_SPLITK");
+    if (env && env[0] == '1') g_allow_splitk = false;
+    env = getenv("SEG_NO_PAIRS");
+    if (env && env[0] == '1') g_allow_pairs = false;
+    env = getenv("SEG_PAIR_MIN_TILES");
+    if (env) g_pair_min_tiles = atol(env);
+    g_init_ok = true;
+  });
   return g_init_ok;
+}
+
+// ---- self-test of the bounded wait ---------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(32)
+wait_selftest_kernel(int* dev_status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // nothing ever arrives at this barrier: the wait below ends only through its own time limit
+    mbar_wait(smem_u32(&bar), 0, &abort_flag, dev_status, limit_ns);
+  }
+}
+}  // namespace
+
+cudaError_t launch_wait_selftest(int* dev_status, uint64_t limit_ns, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(dev_status, limit_ns);
+  return cudaGetLastError();
 }
 
 // The mean-squared-error loss of a non-final segment is fused into the split-K kernel, the one that
@@ -1248,7 +1274,7 @@ bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32) {
   return pick_split(M, N, K, tf32) > 1;
 }
 
-cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
+cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s, int* family) {
   if (!g_init_ok) return cudaErrorNotSupported;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return cudaErrorNotSupported;
   if (g.a_dt != g.b_dt) return cudaErrorNotSupported;
@@ -1292,6 +1318,7 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s) {
   e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
   e.loss = g.loss; e.loss.enabled = fuse_loss ? 1 : 0;
 
+  if (family) *family = pairs ? FAM_TC_PAIR : (split > 1 ? FAM_TC_SPLITK : FAM_TC_SINGLE);
   if (pairs) {
     return tf32 ? launch_pair_majors<true>(a_mn, b_mn, ma, mb, g, e, dev_status, s)
                 : launch_pair_majors<false>(a_mn, b_mn, ma, mb, g, e, dev_status, s);

@@ -26,8 +26,10 @@
 #include <stdlib.h>
 
 #include <algorithm>
+#include <atomic>
 #include <functional>
 #include <map>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -57,7 +59,10 @@ struct seg_handle {
   float lr = 0, momentum = 0, beta1 = 0, beta2 = 0, eps = 0;
   uint64_t init_seed = 0;
   cudaStream_t stream = nullptr;
+  int device = 0;                  // the device the handle lives on (current when seg_create ran)
   bool use_tc = false;
+  bool force_tc = false;           // SEG_GEMM_TCGEN05: a product the tensor-core path cannot take is an error
+  uint64_t family_launches[FAM_COUNT] = {0, 0, 0, 0};
   int act_dt = DT_F32, act_round = RND_NONE, op_dt = DT_F32, op_round = RND_NONE;
   std::vector<int> widths;
   std::vector<LayerInfo> layers;
@@ -89,6 +94,7 @@ struct seg_handle {
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
     uint64_t kernels = 0, kernels_peer = 0;
+    uint64_t family[FAM_COUNT] = {0, 0, 0, 0}, family_peer[FAM_COUNT] = {0, 0, 0, 0};
     seg_handle* peer = nullptr;
     cudaGraphNode_t stage_node = nullptr;
     cudaKernelNodeParams stage_params{};
@@ -125,6 +131,7 @@ struct seg_handle {
   uint64_t mem_current = 0, mem_peak = 0, launches = 0;
   std::vector<void*> allocations;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  cudaEvent_t ev_handoff = nullptr;   // seg_handoff_copy: the copy out of this handle's device is complete
   bool profile = false;
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_used = 0;
@@ -133,6 +140,18 @@ struct seg_handle {
 };
 
 namespace {
+
+// Makes the handle's device current for the duration of one call and restores the caller's.
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(const seg_handle* h) {
+    if (!h) return;
+    if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return; }
+    if (prev != h->device && cudaSetDevice(h->device) == cudaSuccess) switched = true;
+  }
+  ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
 
 seg_status fail_cuda(seg_handle* h, cudaError_t e, const char* what) {
   if (h) h->last_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -196,12 +215,19 @@ seg_status run_gemm(seg_handle* h, const GemmDesc& g_in, int kind, cudaStream_t 
     g.simt_slots = h->simt_slots[workspace];
   }
   if (h->use_tc) {
-    cudaError_t e = launch_gemm_tc(g, h->dev_status, stream);
-    if (e == cudaSuccess) { if (used_tc) *used_tc = true; return SEG_OK; }
+    int family = FAM_TC_SINGLE;
+    cudaError_t e = launch_gemm_tc(g, h->dev_status, stream, &family);
+    if (e == cudaSuccess) { if (used_tc) *used_tc = true; ++h->family_launches[family]; return SEG_OK; }
     if (e != cudaErrorNotSupported) return fail_cuda(h, e, "tensor-core product launch");
     cudaGetLastError();
+    if (h->force_tc) {
+      h->last_error = "the tensor-core path cannot take this product (operand alignment or strides) and the handle "
+                      "was created with SEG_GEMM_TCGEN05";
+      return SEG_ERR_UNSUPPORTED;
+    }
   }
   SEG_TRY(h, launch_gemm_simt(g, stream), "FFMA product launch");
+  ++h->family_launches[FAM_SIMT];
   return SEG_OK;
 }
 
@@ -255,7 +281,7 @@ seg_status launch_loss(seg_handle* h, int batch, const int32_t* cls, float* cons
                                       h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
                                       h->loss_partials, h->loss_counter, loss_dst, h->stream), "softmax-CE loss");
   } else {
-    SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], cls, h->sil, h->widths[L], batch,
+    SEG_TRY(h, launch_mse_loss(h->act[L], h->act_dtype[L], h->ld_act[L], cls, h->sil, h->n_classes, h->widths[L], batch,
                                h->last_relu ? 1 : 0, dz_L, h->act_dt, h->act_round, h->ld_act[L],
                                h->loss_partials, h->loss_counter, loss_dst, h->stream), "MSE loss");
   }
@@ -311,7 +337,7 @@ seg_status refresh_operand_copy(seg_handle* h, int64_t off, int64_t n) {
   if (!h->params_op || n == 0) return SEG_OK;
   Launch l(h, K_COPY);
   char* dst = reinterpret_cast<char*>(h->params_op) + off * elem_size(h->op_dt);
-  SEG_TRY(h, launch_copy2d(dst, h->op_dt, n, h->params + off, DT_F32, n, 1, (int)n, h->op_round,
+  SEG_TRY(h, launch_copy2d(dst, h->op_dt, n, h->params + off, DT_F32, n, 1, n, h->op_round,
                            h->stream), "operand copy refresh");
   return SEG_OK;
 }
@@ -333,6 +359,7 @@ const char* seg_status_string(int32_t s) {
     case SEG_ERR_STATE: return "call not valid in this state";
     case SEG_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait";
     case SEG_ERR_NO_DEVICE: return "no usable CUDA device";
+    case SEG_ERR_CLASS_RANGE: return "class index outside [0, n_classes)";
     default: return "unknown status";
   }
 }
@@ -364,8 +391,10 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
 
   seg_handle* h = new (std::nothrow) seg_handle();
   if (!h) return SEG_ERR_ALLOC;
-  static uint64_t next_uid = 0;
+  static std::atomic<uint64_t> next_uid{0};
   h->uid = ++next_uid;
+  h->device = dev;
+  h->force_tc = cfg->gemm_backend == SEG_GEMM_TCGEN05;
   h->n_layers = cfg->n_layers; h->n_classes = cfg->n_classes; h->max_batch = cfg->max_batch;
   h->segment_id = cfg->segment_id; h->is_final = cfg->is_final != 0;
   h->last_relu = cfg->last_relu < 0 ? !h->is_final : (cfg->last_relu != 0);
@@ -444,8 +473,11 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   {
     const char* env = getenv("SEG_NO_GRAPH");
     if (env && env[0] == '1') h->graphs_enabled = false;
-    env = getenv("SEG_NO_PDL");
-    if (env && env[0] == '1') g_use_pdl = false;
+    static std::once_flag pdl_once;      // process-wide switch: written once, before any launch of any handle
+    std::call_once(pdl_once, [] {
+      const char* e = getenv("SEG_NO_PDL");
+      if (e && e[0] == '1') g_use_pdl = false;
+    });
     env = getenv("SEG_NO_FORK");
     if (env && env[0] == '1') h->fork_enabled = false;
     env = getenv("SEG_NO_FUSED_LOSS");
@@ -496,6 +528,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
 
 seg_status seg_destroy(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
+  if (h->ev_handoff) cudaEventDestroy(h->ev_handoff);
   if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
   cudaStreamSynchronize(h->stream);
   for (cudaStream_t ls : h->lstream) if (ls) cudaStreamSynchronize(ls);
@@ -527,6 +561,7 @@ seg_status seg_destroy(seg_handle* h) {
 
 seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, float kappa) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (h->is_final) return SEG_ERR_STATE;
   if (dist != SEG_LABEL_UNIFORM_KAPPA && dist != SEG_LABEL_NORMAL) return SEG_ERR_INVALID_ARG;
   Launch l(h, K_COPY);
@@ -538,6 +573,7 @@ seg_status seg_gen_labels(seg_handle* h, uint64_t seed, int32_t dist, float kapp
 
 seg_status seg_forward(seg_handle* h, const void* x, int32_t batch, void* y) {
   if (!h || !x || !y) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   seg_status st = forward_impl(h, x, batch);
   if (st != SEG_OK) return st;
@@ -573,7 +609,7 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   gather, loss_to, h->loss_dst, mainst), "input staging");
+                                   gather, loss_to, h->loss_dst, h->n_classes, h->dev_status, mainst), "input staging");
   }
   if (h->capturing) h->cap_stage_node = last_captured_node(h);
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch, h->cls_stage, h->loss_dst)) != SEG_OK) return st;
@@ -644,7 +680,7 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
 }
 
 // Index of the caller-supplied pointers in the kernels' parameter lists (see elementwise.cu).
-static const int kStageArgCount = 17, kStageArgX = 3, kStageArgCls = 9, kStageArgGather = 14, kStageArgLoss = 15;
+static const int kStageArgCount = 19, kStageArgX = 3, kStageArgCls = 9, kStageArgGather = 14, kStageArgLoss = 15;
 
 static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGraph_t graph) {
   if (!h->cap_stage_node) return false;
@@ -670,7 +706,11 @@ static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const vo
   }
   SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
   h->launches += g.kernels;
-  if (g.peer) g.peer->launches += g.kernels_peer;
+  for (int f = 0; f < FAM_COUNT; ++f) h->family_launches[f] += g.family[f];
+  if (g.peer) {
+    g.peer->launches += g.kernels_peer;
+    for (int f = 0; f < FAM_COUNT; ++f) g.peer->family_launches[f] += g.family_peer[f];
+  }
   return SEG_OK;
 }
 
@@ -687,6 +727,16 @@ static seg_status run_step_captured(seg_handle* h, seg_handle::StepGraph& g, seg
     return enqueue(h->fork_enabled);
   }
   const uint64_t before = h->launches, before_peer = peer ? peer->launches : 0;
+  uint64_t fam_before[FAM_COUNT], fam_before_peer[FAM_COUNT] = {0, 0, 0, 0};
+  for (int f = 0; f < FAM_COUNT; ++f) { fam_before[f] = h->family_launches[f]; if (peer) fam_before_peer[f] = peer->family_launches[f]; }
+  auto restore_counts = [&] {          // what a capture "launched" has not run: take it off the counters again
+    h->launches = before;
+    for (int f = 0; f < FAM_COUNT; ++f) h->family_launches[f] = fam_before[f];
+    if (peer) {
+      peer->launches = before_peer;
+      for (int f = 0; f < FAM_COUNT; ++f) peer->family_launches[f] = fam_before_peer[f];
+    }
+  };
   cudaGraph_t graph = nullptr;
   if (cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
@@ -699,9 +749,13 @@ static seg_status run_step_captured(seg_handle* h, seg_handle::StepGraph& g, seg
   cudaError_t e = cudaStreamEndCapture(h->stream, &graph);
   if (st == SEG_OK && e == cudaSuccess && graph != nullptr && adopt_captured_graph(h, g, graph)) {
     g.kernels = h->launches - before;
-    h->launches = before;
+    for (int f = 0; f < FAM_COUNT; ++f) g.family[f] = h->family_launches[f] - fam_before[f];
     g.peer = peer;
-    if (peer) { g.kernels_peer = peer->launches - before_peer; peer->launches = before_peer; }
+    if (peer) {
+      g.kernels_peer = peer->launches - before_peer;
+      for (int f = 0; f < FAM_COUNT; ++f) g.family_peer[f] = peer->family_launches[f] - fam_before_peer[f];
+    }
+    restore_counts();
     return replay_graph(h, g, x, cls, loss_to, gather);
   }
   // capture did not work here: run eagerly from now on
@@ -712,8 +766,7 @@ static seg_status run_step_captured(seg_handle* h, seg_handle::StepGraph& g, seg
   if (graph) cudaGraphDestroy(graph);
   g.exec = nullptr;
   h->graphs_enabled = false;
-  h->launches = before;
-  if (peer) peer->launches = before_peer;
+  restore_counts();
   return enqueue(h->fork_enabled);
 }
 
@@ -723,6 +776,7 @@ static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* c
 seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int32_t batch,
                           float* loss_out, void* y_out) {
   if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   return train_step_impl(h, x, cls, batch, loss_out, y_out, nullptr);
 }
 
@@ -731,6 +785,7 @@ seg_status seg_train_step(seg_handle* h, const void* x, const int32_t* cls, int3
 seg_status seg_train_step_label_input(seg_handle* h, const float* sil_in, const int32_t* cls, int32_t batch,
                                       float* loss_out) {
   if (!h || !sil_in || !cls) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   return train_step_impl(h, nullptr, cls, batch, loss_out, nullptr, sil_in);
 }
 
@@ -747,6 +802,7 @@ static seg_status train_step_impl(seg_handle* h, const void* x, const int32_t* c
   }
   if (st != SEG_OK) return st;
   ++h->step;
+  h->last_batch = batch;           // a replayed graph does not pass through forward_layers
   if (y_out && (st = copy_out(h, y_out, batch)) != SEG_OK) return st;
   return SEG_OK;
 }
@@ -761,7 +817,7 @@ static seg_status enqueue_recovery(seg_handle* h, seg_handle* r, int batch, bool
     Launch lc(h, K_COPY);
     SEG_TRY(h, launch_stage_inputs(h->x_stage, h->act_dt, h->ld_act[0], x, h->widths[0], batch, h->widths[0],
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
-                                   nullptr, loss_to, h->loss_dst, s), "input staging");
+                                   nullptr, loss_to, h->loss_dst, h->n_classes, h->dev_status, s), "input staging");
   }
   if (h->capturing) h->cap_stage_node = last_captured_node(h);
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
@@ -790,6 +846,8 @@ static seg_status enqueue_recovery(seg_handle* h, seg_handle* r, int batch, bool
 seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x, const int32_t* cls,
                              int32_t batch, float* loss_out) {
   if (!left || !right || !x || !cls) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(left);
+  if (left->device != right->device) return SEG_ERR_UNSUPPORTED;    // the joined network runs on one device
   if (batch < 1 || batch > left->max_batch || batch > right->max_batch) return SEG_ERR_SHAPE;
   if (left->is_final || !right->is_final) return SEG_ERR_STATE;
   if (left->widths[left->n_layers] != right->widths[0]) return SEG_ERR_SHAPE;
@@ -815,6 +873,7 @@ seg_status seg_recovery_step(seg_handle* left, seg_handle* right, const void* x,
 seg_status seg_train_epochs(seg_handle* h, const void* x, const int32_t* cls, int64_t n, int32_t batch,
                             int32_t epochs, float* losses) {
   if (!h || !x || !cls) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (n < 1 || epochs < 0) return SEG_ERR_SHAPE;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   const size_t row_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
@@ -832,6 +891,7 @@ seg_status seg_train_epochs(seg_handle* h, const void* x, const int32_t* cls, in
 
 seg_status seg_forward_dataset(seg_handle* h, const void* x, int64_t n, int32_t batch, void* y) {
   if (!h || !x || !y) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (n < 1) return SEG_ERR_SHAPE;
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   const size_t in_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
@@ -857,6 +917,7 @@ static const void* mapped_device_pointer(const void* host) {
 seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t* cls_host, int32_t batch,
                                float* loss_host) {
   if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   seg_status st;
   const size_t row_bytes = (size_t)h->widths[0] * elem_size(h->act_dt);
@@ -896,6 +957,7 @@ seg_status seg_train_step_host(seg_handle* h, const void* x_host, const int32_t*
 seg_status seg_train_step_host_async(seg_handle* h, const void* x_host, const int32_t* cls_host, int32_t batch,
                                      float* loss_host) {
   if (!h || !x_host || !cls_host) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (batch < 1 || batch > h->max_batch) return SEG_ERR_SHAPE;
   if (!mapped_device_pointer(x_host) || !mapped_device_pointer(cls_host)) return SEG_ERR_INVALID_ARG;   // pageable
   float* loss_dev = nullptr;
@@ -934,6 +996,7 @@ seg_status seg_train_step_host_async(seg_handle* h, const void* x_host, const in
 
 seg_status seg_get_labels(seg_handle* h, float* dst) {
   if (!h || !dst) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (h->is_final || !h->have_labels) return SEG_ERR_STATE;
   SEG_TRY(h, cudaMemcpyAsync(dst, h->sil, sizeof(float) * h->n_classes * h->widths[h->n_layers],
                              cudaMemcpyDeviceToDevice, h->stream), "label copy");
@@ -942,6 +1005,7 @@ seg_status seg_get_labels(seg_handle* h, float* dst) {
 
 seg_status seg_set_labels(seg_handle* h, const float* src) {
   if (!h || !src) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (h->is_final) return SEG_ERR_STATE;
   SEG_TRY(h, cudaMemcpyAsync(h->sil, src, sizeof(float) * h->n_classes * h->widths[h->n_layers],
                              cudaMemcpyDeviceToDevice, h->stream), "label copy");
@@ -951,6 +1015,7 @@ seg_status seg_set_labels(seg_handle* h, const float* src) {
 
 static seg_status get_flat(seg_handle* h, const float* base, int layer, float* W, float* b) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
   if (!base) return SEG_ERR_STATE;
   const LayerInfo& L = h->layers[layer];
@@ -972,12 +1037,14 @@ seg_status seg_get_grads(seg_handle* h, int32_t layer, float* dW, float* db) {
 
 seg_status seg_get_opt_state(seg_handle* h, int32_t layer, int32_t which, float* sW, float* sb) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (which != 0 && which != 1) return SEG_ERR_INVALID_ARG;
   return get_flat(h, which == 0 ? h->state1 : h->state2, layer, sW, sb);
 }
 
 seg_status seg_set_opt_state(seg_handle* h, int32_t layer, int32_t which, const float* sW, const float* sb) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (which != 0 && which != 1) return SEG_ERR_INVALID_ARG;
   if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
   float* base = which == 0 ? h->state1 : h->state2;
@@ -999,6 +1066,7 @@ seg_status seg_get_step(const seg_handle* h, uint64_t* step) {
 
 seg_status seg_set_step(seg_handle* h, uint64_t step) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   h->step = step;
   const unsigned long long t = step;
   SEG_TRY(h, cudaMemcpyAsync(h->step_dev, &t, sizeof(t), cudaMemcpyHostToDevice, h->stream), "step counter copy");
@@ -1008,6 +1076,7 @@ seg_status seg_set_step(seg_handle* h, uint64_t step) {
 
 seg_status seg_set_params(seg_handle* h, int32_t layer, const float* W, const float* b) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (!valid_layer(h, layer)) return SEG_ERR_SHAPE;
   const LayerInfo& L = h->layers[layer];
   if (W) {
@@ -1021,6 +1090,7 @@ seg_status seg_set_params(seg_handle* h, int32_t layer, const float* W, const fl
 
 seg_status seg_get_activation(seg_handle* h, int32_t layer, float* dst) {
   if (!h || !dst) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (layer < 1 || layer > h->n_layers) return SEG_ERR_SHAPE;
   if (h->last_batch < 1) return SEG_ERR_STATE;
   Launch l(h, K_COPY);
@@ -1044,31 +1114,80 @@ seg_status seg_launch_count(const seg_handle* h, uint64_t* launches) {
 
 seg_status seg_poll_status(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   int host = 0;
   SEG_TRY(h, cudaMemcpyAsync(&host, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream), "status read");
   SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
   if (host != DEV_OK) {
     cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream);
-    h->last_error = "a kernel gave up a bounded wait";
-    return SEG_ERR_DEVICE_TIMEOUT;
+    if (host & DEV_TIMEOUT) {
+      h->last_error = "a kernel gave up a bounded wait";
+      return SEG_ERR_DEVICE_TIMEOUT;
+    }
+    h->last_error = "a step met a class index outside [0, n_classes); it was clamped";
+    return SEG_ERR_CLASS_RANGE;
   }
+  return SEG_OK;
+}
+
+seg_status seg_product_launches(const seg_handle* h, uint64_t* counts) {
+  if (!h || !counts) return SEG_ERR_INVALID_ARG;
+  for (int f = 0; f < FAM_COUNT; ++f) counts[f] = h->family_launches[f];
+  return SEG_OK;
+}
+
+seg_status seg_device(const seg_handle* h, int32_t* device) {
+  if (!h || !device) return SEG_ERR_INVALID_ARG;
+  *device = h->device;
+  return SEG_OK;
+}
+
+seg_status seg_selftest_bounded_wait(seg_handle* h, uint64_t limit_ns) {
+  if (!h) return SEG_ERR_INVALID_ARG;
+  if (limit_ns < 1000ull || limit_ns > 1000000000ull) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
+  ++h->launches;
+  SEG_TRY(h, launch_wait_selftest(h->dev_status, limit_ns, h->stream), "bounded-wait self-test");
+  return SEG_OK;
+}
+
+// Section 2.1: the only data that ever moves between partitions is the stored response of the previous one.
+seg_status seg_handoff_copy(seg_handle* producer, const void* src, seg_handle* consumer, void* dst, uint64_t bytes) {
+  if (!producer || !consumer || !src || !dst) return SEG_ERR_INVALID_ARG;
+  if (bytes == 0) return SEG_OK;
+  seg_handle* h = producer;
+  DeviceGuard guard(h);
+  if (producer->device == consumer->device) {
+    SEG_TRY(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, producer->stream), "hand-off copy");
+  } else {
+    SEG_TRY(h, cudaMemcpyPeerAsync(dst, consumer->device, src, producer->device, bytes, producer->stream), "hand-off copy");
+  }
+  if (producer->stream == consumer->stream) return SEG_OK;     // one stream: already ordered
+  if (!producer->ev_handoff)
+    SEG_TRY(h, cudaEventCreateWithFlags(&producer->ev_handoff, cudaEventDisableTiming), "event create");
+  SEG_TRY(h, cudaEventRecord(producer->ev_handoff, producer->stream), "event record");
+  DeviceGuard guard_consumer(consumer);
+  SEG_TRY(consumer, cudaStreamWaitEvent(consumer->stream, producer->ev_handoff, 0), "stream wait");
   return SEG_OK;
 }
 
 seg_status seg_timer_start(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   SEG_TRY(h, cudaEventRecord(h->ev_start, h->stream), "event record");
   return SEG_OK;
 }
 
 seg_status seg_timer_stop(seg_handle* h) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   SEG_TRY(h, cudaEventRecord(h->ev_stop, h->stream), "event record");
   return SEG_OK;
 }
 
 seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms) {
   if (!h || !ms) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   SEG_TRY(h, cudaEventSynchronize(h->ev_stop), "event synchronize");
   SEG_TRY(h, cudaEventElapsedTime(ms, h->ev_start, h->ev_stop), "event elapsed");
   return SEG_OK;
@@ -1076,6 +1195,7 @@ seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms) {
 
 seg_status seg_profile_enable(seg_handle* h, int32_t on) {
   if (!h) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
   h->profile = on != 0;
   h->ev_used = 0;
@@ -1085,6 +1205,7 @@ seg_status seg_profile_enable(seg_handle* h, int32_t on) {
 
 seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms) {
   if (!h || !count || !total_ms) return SEG_ERR_INVALID_ARG;
+  DeviceGuard guard(h);
   if (kind < 0 || kind >= K_COUNT) return SEG_ERR_INVALID_ARG;
   SEG_TRY(h, cudaStreamSynchronize(h->stream), "stream synchronize");
   uint64_t n = 0; double total = 0.0;

@@ -9,7 +9,9 @@ import pytest
 
 from oracle import rng as orng
 from paper_2403_11204_b200 import workloads as wl
-from parity_util import (batch_arrays, bits_equal, compare_step, make_pair, rel_err, sync_from_oracle,
+import os
+
+from parity_util import (batch_arrays, bits_equal, compare_step, make_oracle, make_pair, rel_err, sync_from_oracle,
                          to_device)
 
 pytestmark = pytest.mark.gpu
@@ -251,14 +253,178 @@ TC_CASES = [
 ]
 
 
+def expected_families(widths, batch):
+    """Which product-kernel families a step of this shape must / must not launch, given the selection
+    switches this process runs under (the forced-selection child runs set them)."""
+    must, never = set(), {"ffma"}                     # SEG_GEMM_TCGEN05: never the FFMA kernels
+    if os.environ.get("SEG_NO_SPLITK") == "1":
+        never.add("tc_splitk")
+    if os.environ.get("SEG_NO_PAIRS") == "1":
+        never.add("tc_pair")
+    if os.environ.get("SEG_NO_SPLITK") == "1" and os.environ.get("SEG_NO_PAIRS") == "1":
+        must.add("tc_single")
+    if os.environ.get("SEG_PAIR_MIN_TILES") == "1" and os.environ.get("SEG_NO_PAIRS") != "1":
+        # pairs from one 256 x 256 tile on: any product with M, N, K >= 256 that is not split over K
+        if batch >= 256 and min(widths) >= 256 and os.environ.get("SEG_NO_SPLITK") == "1":
+            must.add("tc_pair")
+    return must, never
+
+
 @pytest.mark.parametrize("widths,final,precision,optimizer,batch", TC_CASES)
 def test_single_step_tensor_core_backend(widths, final, precision, optimizer, batch):
     w = wl.WORKLOADS["tiny"]
     gpu, ora = make_pair(widths, 47, final, precision, optimizer, 1e-3, batch, gemm_backend="tcgen05")
+    plain = make_oracle(widths, 47, final, "fp32", optimizer, 1e-3)
     x, cls = batch_arrays(w, batch, widths[0], precision=precision)
-    compare_step(gpu, ora, x, cls, precision, TOL[precision])
+    report = {}
+    compare_step(gpu, ora, x, cls, precision, TOL[precision], ora_plain=plain, report=report)
+    print(widths, precision, {k: v for k, v in report.items() if k != "vs_plain_fp32_oracle"},
+          "vs plain fp32 oracle:", {k: f"{v:.1e}" for k, v in report["vs_plain_fp32_oracle"].items()})
     x2, cls2 = batch_arrays(w, max(batch - 1, 1), widths[0], seed=5, precision=precision)
     if optimizer == "adam":
         sync_from_oracle(gpu, ora)
     compare_step(gpu, ora, x2, cls2, precision, TOL[precision])      # smaller batch on the same handle
+    # which kernels ran: every product of both steps on tensor cores, in the family the switches allow
+    fam = gpu.product_launches()
+    n_products = 2 * (3 * len(widths) - 4)            # per step: L forward, L weight-gradient, L - 1 dgrad products
+    assert sum(fam.values()) == n_products, fam
+    must, never = expected_families(widths, batch)
+    assert all(fam[f] == 0 for f in never), (fam, never)
+    assert all(fam[f] > 0 for f in must), (fam, must)
     gpu.close()
+
+
+def test_product_family_counters_tell_the_backends_apart():
+    """seg_product_launches is what the tensor-core tests rely on to show that tcgen05 kernels ran, so it is
+    checked from both sides: a bf16 handle on the automatic or the tensor-core backend counts its five
+    products (2 forward, 2 weight-gradient, 1 dgrad) as tensor-core launches and none as FFMA; the same
+    segment on the FFMA backend counts all five as FFMA.  (With SEG_GEMM_TCGEN05 a product the tensor-core
+    path could not take would be SEG_ERR_UNSUPPORTED, never an FFMA launch; the handle's own buffers are
+    always laid out so that it can.)"""
+    import torch
+    from paper_2403_11204_b200.binding import Segment
+    x = torch.rand(8, 24, device="cuda").to(torch.bfloat16)
+    cls = torch.zeros(8, dtype=torch.int32, device="cuda")
+    for backend in ("auto", "tcgen05", "simt"):
+        seg = Segment([24, 16, 8], 47, False, precision="bf16", max_batch=8, gemm_backend=backend)
+        seg.gen_labels(1)
+        for _ in range(4):                               # eager, captured and replayed steps all count
+            seg.train_step(x, cls)
+        seg.poll()
+        fam = seg.product_launches()
+        tc = fam["tc_single"] + fam["tc_splitk"] + fam["tc_pair"]
+        assert (fam["ffma"], tc) == ((20, 0) if backend == "simt" else (0, 20)), (backend, fam)
+        seg.close()
+
+
+def test_replayed_step_reports_its_own_batch_size():
+    """A step replayed from its captured graph must leave the handle knowing that step's batch size:
+    seg_get_activation after it copies exactly that many rows (guard rows behind the buffer stay
+    untouched), also when a forward pass at a larger batch ran in between."""
+    import torch
+    w = wl.WORKLOADS["tiny"]
+    A, B = 24, 64
+    gpu, ora = make_pair([784, 128, 64], 47, False, "fp32", "sgd", 0.01, B)
+    x, cls = batch_arrays(w, B, 784)
+    xt, ct = to_device(x, cls, "fp32")
+    for _ in range(3):                                   # eager, capture, replay at batch A
+        gpu.train_step(xt[:A], ct[:A])
+        ora.train_step(x[:A], cls[:A])
+    gpu.forward(xt)                                      # batch B in between
+    gpu.train_step(xt[:A], ct[:A])                       # replayed
+    ora.loss_and_grads(x[:A], cls[:A])
+    buf = torch.full((A + 8, 64), -7.0, device="cuda")   # A rows for the call, 8 guard rows behind them
+    st = gpu.lib.seg_get_activation(gpu.h, 2, buf.data_ptr())
+    assert st == 0
+    gpu.poll()
+    got = buf.cpu().numpy()
+    assert np.all(got[A:] == -7.0), "rows beyond the step's batch were written"
+    assert rel_err(got[:A], ora.acts[2]) < 1e-4
+    gpu.close()
+
+
+def test_bounded_wait_runs_out_and_the_handle_stays_usable():
+    """The product kernels' wait routine, given a barrier nothing arrives at and a limit of one millisecond,
+    gives up, records it, and returns: seg_poll_status reports the time-out once, the next poll is clean,
+    and a training step on the same handle afterwards still matches the oracle."""
+    from paper_2403_11204_b200.binding import SegError
+    w = wl.WORKLOADS["tiny"]
+    gpu, ora = make_pair([64, 128], 47, False, "bf16", "sgd", 0.01, 128, gemm_backend="tcgen05")
+    gpu.selftest_bounded_wait(1_000_000)
+    with pytest.raises(SegError) as e:
+        gpu.poll()
+    assert e.value.status == 7
+    gpu.poll()                                           # the record is cleared by the poll that reported it
+    with pytest.raises(SegError) as e:
+        gpu.selftest_bounded_wait(10)                    # limits outside [1 us, 1 s] are refused
+    assert e.value.status == 1
+    x, cls = batch_arrays(w, 128, 64, precision="bf16")
+    compare_step(gpu, ora, x, cls, "bf16", TOL["bf16"])
+    gpu.close()
+
+
+def test_class_index_out_of_range_is_clamped_and_reported():
+    import torch
+    from paper_2403_11204_b200.binding import SegError
+    w = wl.WORKLOADS["tiny"]
+    gpu, ora = make_pair([64, 64, 32], 47, False, "fp32", "sgd", 0.01, 32)
+    x, cls = batch_arrays(w, 32, 64)
+    bad = cls.copy()
+    bad[3], bad[17] = 47, -5                             # one past the end, one negative
+    xt, ct = to_device(x, bad, "fp32")
+    loss = torch.zeros(1, device="cuda")
+    gpu.train_step(xt, ct, loss)
+    with pytest.raises(SegError) as e:
+        gpu.poll()
+    assert e.value.status == 9
+    clamped = np.clip(bad, 0, 46)
+    ref = ora.train_step(x, clamped)                     # the step that ran is the step on the clamped indices
+    assert abs(float(loss.item()) - ref) / abs(ref) < 1e-4
+    gpu.poll()
+    gpu.close()
+
+
+def test_tie_ceiling_catches_a_widened_band():
+    """The share of ReLU decisions the comparison may take from the CUDA path is bounded: with the band
+    widened a hundredfold the same comparison must fail on that bound."""
+    w = wl.WORKLOADS["tiny"]
+    widths, batch = [784, 320, 200, 72], 300
+    gpu, ora = make_pair(widths, 47, False, "bf16", "sgd", 1e-3, batch, gemm_backend="tcgen05")
+    x, cls = batch_arrays(w, batch, widths[0], precision="bf16")
+    with pytest.raises(AssertionError, match="tie band|large value at a tie|tie decisions"):
+        compare_step(gpu, ora, x, cls, "bf16", TOL["bf16"], tie_scale=100.0)
+    gpu.close()
+
+
+def test_two_segments_hand_off_through_the_library_copy():
+    """Section 2.1 deployment on the devices at hand: each segment is created on a device of its own when
+    the machine has two, otherwise both on device 0 (same code path, the copy is then device-to-device):
+    train the left segment, store its response, hand it to the right segment's device with
+    seg_handoff_copy, train the right segment - against the oracle's procedure."""
+    import torch
+    from oracle import pnn
+    from paper_2403_11204_b200 import binding
+    from paper_2403_11204_b200.binding import Segment
+    from parity_util import make_oracle
+    w = wl.WORKLOADS["tiny"]
+    devs = [0, 1] if torch.cuda.device_count() > 1 else [0, 0]
+    specs = [([784, 64, 32], False), ([32, 32, 47], True)]
+    segs, oras = [], []
+    for k, (widths, final) in enumerate(specs):
+        st = torch.cuda.Stream(device=devs[k])
+        segs.append(Segment(widths, 47, final, precision="fp32", optimizer="momentum", lr=0.01, max_batch=64,
+                            segment_id=k, stream=st, device=devs[k]))
+        oras.append(make_oracle(widths, 47, final, "fp32", "momentum", 0.01, segment_id=k))
+    segs[0].gen_labels(wl.LABEL_SEED, "normal")
+    x, cls = batch_arrays(w, 200, 784)
+    with torch.cuda.device(devs[0]):
+        xt, ct = to_device(x, cls, "fp32")
+    torch.cuda.synchronize()
+    losses, _ = binding.train_partitioned(segs, xt, ct, 64, [2, 2])
+    for s_ in segs:
+        s_.poll()
+    ref, _ = pnn.train_partitioned(oras, x, cls, 64, [2, 2])
+    for got, want in zip(losses, ref):
+        assert np.max(np.abs(got.cpu().numpy() - want) / np.abs(want)) < 1e-3
+    for s_ in segs:
+        s_.close()

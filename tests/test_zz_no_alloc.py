@@ -6,8 +6,10 @@ owns a stream but no allocator): its reduction scratch is a static array inside 
 Here it is fed the stored output, class indices and labels of a real training step and must
 reproduce that step's loss and, through the column sums of its dZ, that step's last-layer bias
 gradient - twice in a row, because the second call meets whatever the first one left in the
-shared scratch.  This file sorts last on purpose: a run that stops at the first failure has
-already run everything else.
+shared scratch.  A second test checks the loss and every element of dZ against the three-line
+formula of the header, written out in NumPy float64, with and without the ReLU mask and for a
+width that the wide (16-byte) code path cannot take.  This file sorts last on purpose: a run that
+stops at the first failure has already run everything else.
 """
 import numpy as np
 import pytest
@@ -54,6 +56,36 @@ def test_noalloc_loss_matches_training_step_twice_in_a_row():
         assert np.max(np.abs(db - ref)) <= TOL * np.max(np.abs(ref))
         assert bool(((dz != 0) <= (out > 0)).all())                  # the ReLU mask of the cut layer
     seg.close()
+
+
+@pytest.mark.parametrize("n_p,batch", [(72, 200), (61, 77), (8, 1)])
+@pytest.mark.parametrize("relu_mask", [1, 0])
+def test_noalloc_loss_matches_its_definition_element_by_element(n_p, batch, relu_mask):
+    """loss = mean (out - sil[cls])^2 and dz = 2 (out - sil[cls]) / (batch n_p) [out > 0 if masked], every
+    element, on two calls in a row; class indices outside [0, n_classes) are clamped, not read out of bounds."""
+    import torch
+    from paper_2403_11204_b200 import build
+    build.build()
+    from paper_2403_11204_b200.binding import label_loss_noalloc
+    g = np.random.default_rng(n_p * 1000 + batch)
+    n_classes = 47
+    sil = g.standard_normal((n_classes, n_p)).astype(np.float32)
+    for call in range(2):
+        out = g.standard_normal((batch, n_p)).astype(np.float32)
+        cls = g.integers(0, n_classes, batch).astype(np.int32)
+        if batch > 2 and call == 1:
+            cls[0], cls[1] = n_classes + 3, -1                       # clamped to the last / first class
+        t = sil[np.clip(cls, 0, n_classes - 1)].astype(np.float64)
+        d = out.astype(np.float64) - t
+        loss_ref = float(np.mean(d * d))
+        dz_ref = 2.0 * d / (batch * n_p) * ((out > 0) if relu_mask else 1.0)
+        out_t, cls_t, sil_t = (torch.from_numpy(a).cuda() for a in (out, cls, sil))
+        dz_t, loss_t = torch.full_like(out_t, 7.0), torch.zeros(1, device="cuda")
+        label_loss_noalloc(out_t, cls_t, sil_t, relu_mask, dz_t, loss_t)
+        torch.cuda.synchronize()
+        assert abs(float(loss_t.item()) - loss_ref) <= TOL * abs(loss_ref)
+        err = np.max(np.abs(dz_t.cpu().numpy().astype(np.float64) - dz_ref))
+        assert err <= TOL * np.max(np.abs(dz_ref)), (call, err)
 
 
 def test_noalloc_rejects_sizes_beyond_its_maximum():
