@@ -378,22 +378,36 @@ def _rank_barrier():
 
 
 def kernel_breakdown(r, steps, first, peaks):
-    """Per-kind device time: the same steps again with CUDA events around every launch (one stream, so the
-    kinds add up to the serial time of a step).  Returns (kernels dict, roofline dict of the dominant kind)."""
+    """Per-kind device time: the same steps again, one segment at a time, with CUDA events around every launch
+    on the segment's stream (so the kinds add up to the serial time of the step).  Where weight-gradient
+    products also apply the optimizer update (seg_profile_get kind 4), the weight-gradient and update kinds
+    are reported as one kind, `wgrad_update`, with the products' FLOPs and the update's bytes beside its time.
+    Returns (kernels dict, roofline dict of the dominant kind)."""
     w = r.w
-    for seg in r.segs:
-        seg.profile(True)
-    r.run_steps(first, steps)
-    r.torch.cuda.synchronize()
     kinds = {}
-    for spec, seg in zip(w.segments, r.segs):
+    for k_seg, (spec, seg) in enumerate(zip(w.segments, r.segs)):
+        seg.profile(True)
+        r.run_steps(first, steps, which=k_seg)
+        r.torch.cuda.synchronize()
         work = segment_work(spec, w.batch, w.precision, w.optimizer)
-        for name, (n, tot) in seg.profile_read().items():
-            k = kinds.setdefault(name, {"launches": 0, "ms": 0.0, "flops": 0.0, "bytes": 0.0})
+        prof = seg.profile_read()
+        fused = prof.get("wgrad_update_gemm", (0, 0.0))[0] > 0
+        for name, (n, tot) in prof.items():
+            if fused and name in ("wgrad_gemm", "wgrad_update_gemm", "update"):
+                name = "wgrad_update"
+            elif name == "wgrad_update_gemm":
+                continue
+            k = kinds.setdefault(name, {"launches": 0, "ms": 0.0, "flops": 0.0, "bytes": 0.0, "seen": set()})
             k["launches"] += n
             k["ms"] += tot
+            if (k_seg, name) in k["seen"]:
+                continue
+            k["seen"].add((k_seg, name))
             if name in ("fwd_gemm", "dgrad_gemm", "wgrad_gemm"):
                 k["flops"] += work[name] * steps
+            elif name == "wgrad_update":
+                k["flops"] += work["wgrad_gemm"] * steps
+                k["bytes"] += (work["update_bytes"] + work["bias_grad_bytes"]) * steps
             elif name == "update":          # the update launch also reads dZ for the bias gradient
                 k["bytes"] += (work["update_bytes"] + work["bias_grad_bytes"]) * steps
             elif name == "loss":
@@ -411,9 +425,12 @@ def kernel_breakdown(r, steps, first, peaks):
         if v["flops"] > 0:
             e["tflops"] = round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2)
             e["frac_of_peak"] = round(e["tflops"] / tp, 4)
-        elif v["bytes"] > 0:
+        if v["bytes"] > 0:
             e["gbs"] = round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1)
-            e["frac_of_peak"] = round(e["gbs"] / peaks["hbm_gbs"], 4)
+            if v["flops"] > 0:       # products carrying the update: time against FLOPs at the tensor peak + bytes at the copy bandwidth
+                e["frac_of_sum_roofline"] = round((v["flops"] / (tp * 1e12) + v["bytes"] / (peaks["hbm_gbs"] * 1e9)) / (v["ms"] * 1e-3), 4)
+            else:
+                e["frac_of_peak"] = round(e["gbs"] / peaks["hbm_gbs"], 4)
         kernels[n] = e
     dom = max(kinds, key=lambda n: kinds[n]["ms"])
     v = kinds[dom]
@@ -427,6 +444,10 @@ def kernel_breakdown(r, steps, first, peaks):
                 "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
                 "peak_source": f"{peaks['source']} ({prec_note})", "timing": timing,
                 "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
+        if v["bytes"] > 0:
+            roof["note"] = ("these launches are weight-gradient products whose extra warps also stream the optimizer update "
+                            f"({v['bytes'] / v['launches'] / 1e6:.1f} MB per launch on average, bias update launches included in "
+                            "the time); achieved counts the products' FLOPs only")
     else:
         achieved = v["bytes"] / (v["ms"] * 1e-3) / 1e9
         roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -699,8 +720,8 @@ def main():
                  "precision": ow.precision, "batch": ow.batch, "step": {kk: round(v, 4) for kk, v in r["step"].items()},
                  "segments": short_segments(r["segments"]),
                  "roofline": {kk: r["roofline"][kk] for kk in ("kernel", "bound", "achieved", "peak", "unit", "frac")},
-                 "kernels": {kk: {"share": v["share"], "avg_us": v["avg_us"], "frac_of_peak": v.get("frac_of_peak")}
-                             for kk, v in r["kernels"].items()},
+                 "kernels": {kk: {k2: v[k2] for k2 in ("share", "avg_us", "tflops", "gbs", "frac_of_peak", "frac_of_sum_roofline")
+                                  if k2 in v} for kk, v in r["kernels"].items()},
                  "product_launches": r["product_launches"]}
             if "memory" in r and "ratio" in r["memory"]:
                 o["memory"] = {kk: r["memory"][kk] for kk in ("largest_segment_bytes", "unpartitioned_bytes", "ratio",

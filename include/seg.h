@@ -34,6 +34,8 @@
  *   SEG_NO_PDL=1          ordinary launches instead of programmatic dependent launches
  *   SEG_NO_FUSED_LOSS=1   always run the intermediate-label loss as a launch of its own (default: inside
  *                         the last forward product's epilogue where the tensor-core path can take it)
+ *   SEG_FUSED_UPDATE=1    apply the optimizer update inside the weight-gradient product where a persistent
+ *                         tensor-core kernel runs it (default: a launch of its own, which measured faster)
  *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
  *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
  *   SEG_PAIR_MIN_TILES=n  use CTA pairs exactly when a product has n or more tiles of 256 x 256
@@ -244,9 +246,10 @@ SEG_API seg_status seg_mem_bytes(const seg_handle* h, uint64_t* current, uint64_
 /* Number of kernels the handle has launched so far (host counter). */
 SEG_API seg_status seg_launch_count(const seg_handle* h, uint64_t* launches);
 
-/* Matrix-product launches of this handle so far, by kernel family (host counters; counts[4], host):
+/* Matrix-product launches of this handle so far, by kernel family (host counters; counts[5], host):
  *   [0] tensor-core, one CTA per tile      [1] tensor-core, K split over a cluster
  *   [2] tensor-core, CTA pair per tile     [3] FFMA
+ *   [4] of [0] and [2]: weight-gradient products that also applied the optimizer update
  * Tests use it to show which kernels actually ran.                                           */
 SEG_API seg_status seg_product_launches(const seg_handle* h, uint64_t* counts);
 
@@ -286,8 +289,9 @@ SEG_API seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms);
  * bracketed by CUDA events on the handle's stream.  seg_profile_get synchronises and
  * returns, for one kernel kind, the number of launches and their summed device time
  * since profiling was enabled; kinds: 0 forward product, 1 dgrad product, 2 wgrad
- * product, 3 loss, 4 unused (always 0 launches), 5 optimizer update (forms the bias gradient
- * too), 6 copies / staging.  count and
+ * product, 3 loss, 4 wgrad product that also applies the optimizer update to the weights,
+ * 5 optimizer update as a launch of its own (forms the bias gradient too; after a kind-4
+ * product it has only the bias left), 6 copies / staging.  count and
  * total_ms are host pointers.                                                            */
 SEG_API seg_status seg_profile_enable(seg_handle* h, int32_t on);
 SEG_API seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms);

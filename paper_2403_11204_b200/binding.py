@@ -20,10 +20,10 @@ PRECISIONS = {"fp32": SEG_FP32, "tf32": SEG_TF32, "bf16": SEG_BF16}
 OPTIMIZERS = {"sgd": SEG_SGD, "momentum": SEG_SGD_MOMENTUM, "adam": SEG_ADAM}
 LABEL_DISTS = {"uniform_kappa": SEG_LABEL_UNIFORM_KAPPA, "normal": SEG_LABEL_NORMAL}
 BACKENDS = {"auto": SEG_GEMM_AUTO, "simt": SEG_GEMM_SIMT, "tcgen05": SEG_GEMM_TCGEN05}
-# kind numbers of seg_profile_get (4 is unused: the update launch forms the bias gradient)
-KERNEL_KINDS = {0: "fwd_gemm", 1: "dgrad_gemm", 2: "wgrad_gemm", 3: "loss", 5: "update", 6: "copy"}
-# order of the counters seg_product_launches returns
-PRODUCT_FAMILIES = ("tc_single", "tc_splitk", "tc_pair", "ffma")
+# kind numbers of seg_profile_get
+KERNEL_KINDS = {0: "fwd_gemm", 1: "dgrad_gemm", 2: "wgrad_gemm", 3: "loss", 4: "wgrad_update_gemm", 5: "update", 6: "copy"}
+# order of the counters seg_product_launches returns (the last one counts a subset of tc_single + tc_pair)
+PRODUCT_FAMILIES = ("tc_single", "tc_splitk", "tc_pair", "ffma", "fused_update")
 
 
 class seg_config(Structure):
@@ -164,6 +164,36 @@ def train_partitioned(segments, x, cls, batch, epochs):
                 cur_cls = cur_cls.to(f"cuda:{nxt.device}")
             cur = resp
     return losses, cur
+
+
+def train_partitioned_ranks(seg, x, cls, batch, epochs, rank, world, n_samples=None):
+    """The same procedure with one partition per process (one rank per GPU, torch.distributed already
+    initialised; Section 2.1: each partition trains within its own GPU and the only transfer is the
+    previous partition's stored response, once).  Rank k owns segment k (`seg`), trains it for `epochs`
+    passes and sends its stored response to rank k + 1 as ONE point-to-point message; rank 0 reads x,
+    later ranks receive their input (x is ignored there and may be None).  cls, the class indices, must
+    be present on every rank (they are labels of the data set, not something a partition computes).
+    There is no collective and nothing else crosses between ranks.  `seg` needs train_epochs(x, cls,
+    batch, epochs, losses), forward_dataset(x, batch), widths and act_dtype, which Segment provides.
+    Returns (per-step losses of this rank's segment, this rank's input)."""
+    import torch
+    import torch.distributed as dist
+    n = int(cls.shape[0] if n_samples is None else n_samples)
+    if rank == 0:
+        cur = x
+    else:
+        cur = torch.empty(n, seg.widths[0], dtype=seg.act_dtype, device=cls.device)
+        dist.recv(cur, src=rank - 1)                    # the one transfer into this partition
+    steps = epochs * (-(-n // batch))
+    losses = torch.zeros(max(steps, 1), dtype=torch.float32, device=cls.device)
+    seg.train_epochs(cur, cls, batch, epochs, losses)
+    if rank + 1 < world:
+        resp = seg.forward_dataset(cur, batch)
+        if resp.is_cuda:
+            torch.cuda.current_stream(resp.device).synchronize()
+            seg.stream.synchronize()                    # the response is complete before it leaves the device
+        dist.send(resp.contiguous(), dst=rank + 1)
+    return losses[:steps], cur
 
 
 def recovery_step(left, right, x, cls, loss_out=None):
@@ -371,7 +401,7 @@ class Segment:
 
     def product_launches(self):
         """seg_product_launches as a dict: launches per product-kernel family."""
-        c = (c_uint64 * 4)()
+        c = (c_uint64 * 5)()
         self._check(self.lib.seg_product_launches(self.h, c), "seg_product_launches")
         return dict(zip(PRODUCT_FAMILIES, (int(v) for v in c)))
 

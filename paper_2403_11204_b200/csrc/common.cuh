@@ -48,6 +48,23 @@ struct LossFuse {
   float* const* loss_dst;   // device slot holding the address that receives the loss
 };
 
+// The optimizer update of a layer's weights applied inside its weight-gradient product (tensor-core
+// persistent kernels only): extra warps of every CTA stream over each output tile once the epilogue
+// warps have stored it, so that the update's HBM traffic runs under the main loop of the following
+// tiles instead of after the product.  All pointers address the layer's weight tensor, laid out as
+// the product's C: element (m, n) at base + m * ldc + n.
+struct FusedUpdate {
+  int enabled;              // 0: plain product
+  float* p;                 // fp32 master weights
+  float* s1;                // momentum buffer / Adam first moment (null for plain SGD)
+  float* s2;                // Adam second moment (null otherwise)
+  void* p_op;               // reduced-precision operand copy of the weights (never null on this path)
+  int op_dt, op_round;      // DType / Round of p_op
+  int optimizer;            // seg_optimizer
+  float lr, momentum, beta1, beta2, eps;
+  const float* bc;          // device: {1-b1^t, 1-b2^t}
+};
+
 // One matrix product  C[M][N] = sum_k A(m,k) * B(k,n)  with explicit element strides, so that
 // forward (A W^T), dgrad (dZ W) and wgrad (dZ^T A) are all expressed by one description.
 struct GemmDesc {
@@ -64,6 +81,7 @@ struct GemmDesc {
   const void* mask;         // EPI_MASK: [M][ldmask] of c_dt
   int64_t ldmask;
   LossFuse loss;            // EPI_BIAS_ACT only
+  FusedUpdate upd;          // EPI_PLAIN (weight gradient) only
   int off_critical_path;    // 1: the product runs beside others (a weight gradient on its branch): the tiling is
                             // chosen for latency plus the SM time it takes away from them, not for latency alone
   // FFMA path only: workspace for splitting K over several CTAs of one tile (may be null: no split).
@@ -86,6 +104,9 @@ bool gemm_tc_init();   // resolves the driver entry point needed for tensor maps
 cudaError_t launch_wait_selftest(int* dev_status, uint64_t limit_ns, cudaStream_t s);
 // True when launch_gemm_tc would take the intermediate-label loss into the forward product M x N x K.
 bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32);
+// True when launch_gemm_tc would run this weight-gradient product (both operands MN-major, EPI_PLAIN) in a
+// persistent kernel that can apply the optimizer update as well (g.upd is not looked at).
+bool gemm_tc_can_fuse_update(const GemmDesc& g);
 
 cudaError_t launch_gen_labels(float* dst, int n_classes, int n_p, uint64_t seed, int segment_id,
                               int dist, float kappa, cudaStream_t s);
@@ -161,6 +182,25 @@ inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// ---- optimizer step on one element ------------------------------------------------------------
+// Section 3: SGD with momentum; plain SGD and Adam as well.  H supplies lr, momentum, beta1, beta2, eps.
+template <int OPT, typename H>
+__device__ __forceinline__ void opt_step(float& p, float g, float& m, float& v, const H& u,
+                                         float inv_bc1, float inv_bc2) {
+  if constexpr (OPT == SEG_SGD) {
+    p = p - u.lr * g;
+  } else if constexpr (OPT == SEG_SGD_MOMENTUM) {
+    m = u.momentum * m + g;
+    p = p - u.lr * m;
+  } else {
+    m = u.beta1 * m + (1.0f - u.beta1) * g;
+    v = u.beta2 * v + (1.0f - u.beta2) * g * g;
+    const float mhat = m * inv_bc1;
+    const float vhat = v * inv_bc2;
+    p = p - u.lr * mhat / (sqrtf(vhat) + u.eps);
+  }
 }
 
 // ---- small device helpers ------------------------------------------------------------------

@@ -182,24 +182,6 @@ softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* _
   finish_loss(bt, partials, counter, loss_out, loss_dst, inv_b, red);
 }
 
-// One optimizer step on one element (Section 3: SGD with momentum; plain SGD and Adam as well).
-template <int OPT>
-__device__ __forceinline__ void opt_step(float& p, float g, float& m, float& v, const UpdateArgs& u,
-                                         float inv_bc1, float inv_bc2) {
-  if constexpr (OPT == SEG_SGD) {
-    p = p - u.lr * g;
-  } else if constexpr (OPT == SEG_SGD_MOMENTUM) {
-    m = u.momentum * m + g;
-    p = p - u.lr * m;
-  } else {
-    m = u.beta1 * m + (1.0f - u.beta1) * g;
-    v = u.beta2 * v + (1.0f - u.beta2) * g * g;
-    const float mhat = m * inv_bc1;
-    const float vhat = v * inv_bc2;
-    p = p - u.lr * mhat / (sqrtf(vhat) + u.eps);
-  }
-}
-
 // The update of one layer in one launch.  Parameters, gradients and optimizer state share one flat
 // layout [W | b]:
 //   blocks [0, bias_blocks): each forms the bias gradient of 8 or 32 columns, db[n] = sum_b dZ[b][n]
@@ -453,7 +435,9 @@ cudaError_t launch_update(const UpdateArgs& u, cudaStream_t s) {
   const int bias_cols = (u.batch <= 1024 || u.n_bias <= 256) ? 8 : 32;   // narrow layers: few blocks either way, keep the walk short
   const int bias_blocks = (u.dz != nullptr && u.n_bias > 0) ? (u.n_bias + bias_cols - 1) / bias_cols : 0;
   if (u.n == 0 && bias_blocks == 0) return cudaSuccess;
-  const int grid = bias_blocks + (u.n > 0 ? grid_for(u.n >> 2, 256, 148 * 8) : 0);
+  // two rounds of resident blocks (8 per SM): measured 5.6 TB/s against 4.9 with one round on the 67 M-element
+  // momentum update, no difference for Adam; streaming (evict-first) loads and stores measured no better
+  const int grid = bias_blocks + (u.n > 0 ? grid_for(u.n >> 2, 256, 148 * 16) : 0);
   const bool bf = (u.p_op != nullptr && u.op_dt == DT_BF16);
 #define SEGK_UPD(OPT)                                                      \
   if (bf) launch_k(update_kernel<OPT, DT_BF16>, dim3(grid), dim3(256), 0, s, u, bias_blocks, bias_cols);             \

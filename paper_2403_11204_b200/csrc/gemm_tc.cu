@@ -50,7 +50,9 @@ namespace {
 constexpr int BLOCK_M = 128;
 constexpr int TILE_ROW_BYTES = 128;                    // one swizzle row
 constexpr int A_TILE_BYTES = BLOCK_M * TILE_ROW_BYTES; // 16 KiB per stage
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 192;                       // TMA warp, MMA warp, four epilogue warps
+constexpr int UPDATE_WARPS = 8;                        // fused-update variants: eight more warps stream the optimizer update
+constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * UPDATE_WARPS;
 constexpr int SMEM_BUDGET = 192 * 1024;                // operand ring
 constexpr int SMEM_EXTRA = 2048;                       // alignment slack + barriers
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
@@ -176,6 +178,7 @@ struct EpilogueArgs {
   const void* mask;
   int64_t ldmask;
   LossFuse loss;
+  FusedUpdate upd;
 };
 
 template <int BLOCK_N>
@@ -413,8 +416,113 @@ __device__ __forceinline__ void loss_finish(const LossFuse& l, float lacc, int q
   }
 }
 
-template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// ---- optimizer update fused into the weight-gradient product ------------------------------------
+// Epilogue warps -> update warps of the same CTA: "one more warp has stored its part of a tile".  The
+// stores are fenced to device scope before the count moves, the update warps read the gradient with
+// L2 loads, so they see it.  The wait is bounded like every other wait of these kernels.
+__device__ __forceinline__ void tile_stored_signal(unsigned int* tiles_done, int lane) {
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) atomicAdd(tiles_done, 1u);
+}
+__device__ __forceinline__ bool tile_stored_wait(volatile unsigned int* tiles_done, unsigned int needed,
+                                                 volatile int* abort_flag, int* dev_status, int lane) {
+  int ok = 1;
+  if (lane == 0) {
+    uint32_t spins = 0;
+    uint64_t t0 = 0;
+    while (*tiles_done < needed) {
+      if ((++spins & 0x3Fu) == 0u) {
+        if (*abort_flag) { ok = 0; break; }
+        const uint64_t now = global_timer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > WAIT_LIMIT_NS) {
+          *abort_flag = 1;
+          atomicOr(dev_status, (int)DEV_TIMEOUT);
+          ok = 0;
+          break;
+        }
+        __nanosleep(200);
+      }
+    }
+  }
+  ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+  __threadfence();
+  return ok != 0;
+}
+
+__device__ __forceinline__ void opt_apply(const FusedUpdate& f, float& p, float g, float& m, float& v,
+                                          float inv_bc1, float inv_bc2) {
+  switch (f.optimizer) {
+    case SEG_SGD: opt_step<SEG_SGD>(p, g, m, v, f, inv_bc1, inv_bc2); break;
+    case SEG_SGD_MOMENTUM: opt_step<SEG_SGD_MOMENTUM>(p, g, m, v, f, inv_bc1, inv_bc2); break;
+    default: opt_step<SEG_ADAM>(p, g, m, v, f, inv_bc1, inv_bc2); break;
+  }
+}
+
+// The update of the 128 x TILE_N block of the weight tensor whose gradient sits at g (row pitch ld, as the
+// master weights, the optimizer state and the operand copy), rows m0.., columns n0..  Eight warps; a lane
+// handles four consecutive columns per access (16 bytes; padding columns up to the pitch hold zeros on
+// every side and stay zero), consecutive lanes consecutive groups, and four such groups are in flight per
+// lane before the first is used.  Everything is touched once per step: streaming loads and stores, so that
+// the operand tiles of the product keep their place in L2.
+template <int TILE_N>
+__device__ __forceinline__ void update_tile(const FusedUpdate& f, const float* g, int64_t ld, int m0, int n0,
+                                            int M, int N, int uw, int lane, float inv_bc1, float inv_bc2) {
+  constexpr int VPR = TILE_N / 4;                      // 16-byte groups per tile row
+  constexpr int TOTAL = BLOCK_M * VPR;
+  constexpr int R = 4;
+  constexpr int STRIDE = UPDATE_WARPS * 32;
+  const int n_lim = (N + 3) & ~3;                      // <= ld
+  const bool adam = f.optimizer == SEG_ADAM, mom = f.optimizer != SEG_SGD;
+  for (int base = uw * 32 + lane; base < TOTAL; base += STRIDE * R) {
+    float4 G[R], P[R], S1[R], S2[R];
+    int64_t off[R];
+    bool ok[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      const int v = base + i * STRIDE;
+      const int row = m0 + v / VPR, c = n0 + (v % VPR) * 4;
+      ok[i] = (v < TOTAL) && (row < M) && (c < n_lim);
+      off[i] = (int64_t)row * ld + c;
+      if (ok[i]) {
+        G[i] = __ldcg(reinterpret_cast<const float4*>(g + off[i]));
+        P[i] = __ldcs(reinterpret_cast<const float4*>(f.p + off[i]));
+        if (mom) S1[i] = __ldcs(reinterpret_cast<const float4*>(f.s1 + off[i]));
+        if (adam) S2[i] = __ldcs(reinterpret_cast<const float4*>(f.s2 + off[i]));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      if (!ok[i]) continue;
+      float pv[4] = {P[i].x, P[i].y, P[i].z, P[i].w};
+      const float gv[4] = {G[i].x, G[i].y, G[i].z, G[i].w};
+      float mv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
+      if (mom) { mv[0] = S1[i].x; mv[1] = S1[i].y; mv[2] = S1[i].z; mv[3] = S1[i].w; }
+      if (adam) { vv[0] = S2[i].x; vv[1] = S2[i].y; vv[2] = S2[i].z; vv[3] = S2[i].w; }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) opt_apply(f, pv[k], gv[k], mv[k], vv[k], inv_bc1, inv_bc2);
+      if (mom) __stcs(reinterpret_cast<float4*>(f.s1 + off[i]), make_float4(mv[0], mv[1], mv[2], mv[3]));
+      if (adam) __stcs(reinterpret_cast<float4*>(f.s2 + off[i]), make_float4(vv[0], vv[1], vv[2], vv[3]));
+      __stcs(reinterpret_cast<float4*>(f.p + off[i]), make_float4(pv[0], pv[1], pv[2], pv[3]));
+      if (f.op_dt == DT_BF16) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(pv[0], pv[1]);
+        __nv_bfloat162 hi = __floats2bfloat162_rn(pv[2], pv[3]);
+        uint2 packed;
+        packed.x = *reinterpret_cast<uint32_t*>(&lo);
+        packed.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(f.p_op) + off[i]) = packed;
+      } else {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(f.p_op) + off[i]) =
+            make_float4(apply_round(pv[0], f.op_round), apply_round(pv[1], f.op_round),
+                        apply_round(pv[2], f.op_round), apply_round(pv[3], f.op_round));
+      }
+    }
+  }
+}
+
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N, bool FUSED = false>
+__global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                int M, int N, int K, EpilogueArgs epi, int* dev_status) {
   using L = SmemLayout<BLOCK_N>;
@@ -433,6 +541,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned int* tiles_done = reinterpret_cast<unsigned int*>(tmem_slot + 2);   // FUSED: epilogue-warp arrivals
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar_base = smem_u32(bars);
@@ -447,6 +556,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     *abort_flag = 0;
+    *tiles_done = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -534,7 +644,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
-  } else {
+  } else if (warp < NUM_THREADS / 32) {
     // ---------------- epilogue warps ----------------
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. +31 belong to this warp
     int acc = 0; uint32_t acc_phase = 0;
@@ -559,7 +669,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if constexpr (FUSED) tile_stored_signal(tiles_done, lane);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else if constexpr (FUSED) {
+    // ---------------- update warps: the optimizer on every tile this CTA has stored ----------------
+    if (warp >= NUM_THREADS / 32) {
+      const int uw = warp - NUM_THREADS / 32;
+      float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
+      if (epi.upd.optimizer == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(epi.upd.bc); inv_bc2 = 1.0f / __ldg(epi.upd.bc + 1); }
+      unsigned int needed = 0;
+      for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        needed += 4u;
+        if (!tile_stored_wait(tiles_done, needed, abort_flag, dev_status, lane)) break;
+        const int m0 = (t % tiles_m) * BLOCK_M, n0 = (t / tiles_m) * BLOCK_N;
+        update_tile<BLOCK_N>(epi.upd, reinterpret_cast<const float*>(epi.C), epi.ldc, m0, n0, M, N, uw, lane,
+                             inv_bc1, inv_bc2);
+      }
     }
   }
 
@@ -849,8 +975,8 @@ constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_BYTES;         // 32 KiB 
 constexpr int PAIR_STAGES = 6;
 constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + SMEM_EXTRA;
 
-template <bool TF32, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <bool TF32, bool A_MN, bool B_MN, bool FUSED = false>
+__global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     int M, int N, int K, EpilogueArgs epi, int* dev_status) {
   constexpr int STAGES = PAIR_STAGES;
@@ -868,6 +994,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   // bars[0..S) full (used in the even CTA), [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty (even CTA)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned int* tiles_done = reinterpret_cast<unsigned int*>(tmem_slot + 2);   // FUSED: epilogue-warp arrivals
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();             // 0: issues the MMAs of the pair
@@ -883,6 +1010,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }   // 4 warps x 2 CTAs
     *abort_flag = 0;
+    *tiles_done = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -973,7 +1101,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
-  } else {
+  } else if (warp < NUM_THREADS / 32) {
     // ---------------- epilogue warps: each CTA drains its own 128 rows ----------------
     const int quarter = warp & 3;
     int acc = 0; uint32_t acc_phase = 0;
@@ -999,7 +1127,24 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+      if constexpr (FUSED) tile_stored_signal(tiles_done, lane);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else if constexpr (FUSED) {
+    // ---------------- update warps: the optimizer on this CTA's 128 rows of every tile of the pair ----------------
+    if (warp >= NUM_THREADS / 32) {
+      const int uw = warp - NUM_THREADS / 32;
+      float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
+      if (epi.upd.optimizer == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(epi.upd.bc); inv_bc2 = 1.0f / __ldg(epi.upd.bc + 1); }
+      unsigned int needed = 0;
+      for (int t = pair; t < n_tiles; t += n_pairs) {
+        needed += 4u;
+        if (!tile_stored_wait(tiles_done, needed, abort_flag, dev_status, lane)) break;
+        const int m0 = (t % tiles_m) * PAIR_TILE_M + (int)rank * BLOCK_M;
+        const int n0 = (t / tiles_m) * PAIR_TILE_N;
+        update_tile<PAIR_TILE_N>(epi.upd, reinterpret_cast<const float*>(epi.C), epi.ldc, m0, n0, M, N, uw, lane,
+                                 inv_bc1, inv_bc2);
+      }
     }
   }
 
@@ -1052,6 +1197,7 @@ std::once_flag g_init_once;
 bool g_init_ok = false;
 bool g_allow_splitk = true;
 bool g_allow_pairs = true;
+bool g_allow_fused_update = true;
 long g_pair_min_tiles = 0;      // SEG_PAIR_MIN_TILES: CTA pairs exactly from this many 256 x 256 tiles on (0: cost model)
 
 // 2-D tensor map over a row-major matrix: `inner` contiguous elements per row, `outer` rows,
@@ -1071,16 +1217,17 @@ bool make_map(CUtensorMap* map, bool f32, const void* base, uint64_t inner, uint
   return r == CUDA_SUCCESS;
 }
 
-template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N>
+template <bool TF32, bool A_MN, bool B_MN, int BLOCK_N, bool FUSED = false>
 cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                            const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   using L = SmemLayout<BLOCK_N>;
-  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N>;
+  auto kern = gemm_tc_kernel<TF32, A_MN, B_MN, BLOCK_N, FUSED>;
   static std::atomic<bool> attr_set_dev[kMaxDevices];      // the attribute is per device
   if (cudaError_t err = ensure_dynamic_smem(kern, L::TOTAL, attr_set_dev); err != cudaSuccess) return err;
   const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + BLOCK_N - 1) / BLOCK_N);
   const int grid = tiles < num_sms() ? tiles : num_sms();
-  return launch_k(kern, dim3(grid), dim3(NUM_THREADS), L::TOTAL, s, ma, mb, g.M, g.N, g.K, e, dev_status);
+  return launch_k(kern, dim3(grid), dim3(FUSED ? NUM_THREADS_FUSED : NUM_THREADS), L::TOTAL, s, ma, mb, g.M, g.N, g.K, e,
+                  dev_status);
 }
 
 template <bool TF32, int BLOCK_N>
@@ -1088,7 +1235,10 @@ cudaError_t launch_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUt
                           const GemmDesc& g, const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   if (!a_mn && !b_mn) return launch_variant<TF32, false, false, BLOCK_N>(ma, mb, g, e, dev_status, s);
   if (!a_mn && b_mn) return launch_variant<TF32, false, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
-  if (a_mn && b_mn) return launch_variant<TF32, true, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  if (a_mn && b_mn) {
+    if (e.upd.enabled) return launch_variant<TF32, true, true, BLOCK_N, true>(ma, mb, g, e, dev_status, s);
+    return launch_variant<TF32, true, true, BLOCK_N>(ma, mb, g, e, dev_status, s);
+  }
   return cudaErrorNotSupported;
 }
 
@@ -1142,17 +1292,17 @@ int pick_split(int M, int N, int K, bool tf32) {
   return best;
 }
 
-template <bool TF32, bool A_MN, bool B_MN>
+template <bool TF32, bool A_MN, bool B_MN, bool FUSED = false>
 cudaError_t launch_pair_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
                                 const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
-  auto kern = gemm_tc_pair_kernel<TF32, A_MN, B_MN>;
+  auto kern = gemm_tc_pair_kernel<TF32, A_MN, B_MN, FUSED>;
   static std::atomic<bool> attr_set_dev[kMaxDevices];      // the attribute is per device
   if (cudaError_t err = ensure_dynamic_smem(kern, PAIR_SMEM, attr_set_dev); err != cudaSuccess) return err;
   const int tiles = ((g.M + PAIR_TILE_M - 1) / PAIR_TILE_M) * ((g.N + PAIR_TILE_N - 1) / PAIR_TILE_N);
   const int pairs = std::min(tiles, num_sms() / 2);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = PAIR_SMEM;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
@@ -1169,7 +1319,10 @@ cudaError_t launch_pair_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, cons
                                const GemmDesc& g, const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
   if (!a_mn && !b_mn) return launch_pair_variant<TF32, false, false>(ma, mb, g, e, dev_status, s);
   if (!a_mn && b_mn) return launch_pair_variant<TF32, false, true>(ma, mb, g, e, dev_status, s);
-  if (a_mn && b_mn) return launch_pair_variant<TF32, true, true>(ma, mb, g, e, dev_status, s);
+  if (a_mn && b_mn) {
+    if (e.upd.enabled) return launch_pair_variant<TF32, true, true, true>(ma, mb, g, e, dev_status, s);
+    return launch_pair_variant<TF32, true, true>(ma, mb, g, e, dev_status, s);
+  }
   return cudaErrorNotSupported;
 }
 
@@ -1274,6 +1427,22 @@ bool gemm_tc_can_fuse_loss(int M, int N, int K, bool tf32) {
   return pick_split(M, N, K, tf32) > 1;
 }
 
+// The fused update lives in the persistent kernels (one CTA or a CTA pair per tile); products small enough to
+// be split over K keep the separate update launch, and so does anything the tensor-core path cannot take.
+bool gemm_tc_can_fuse_update(const GemmDesc& g) {
+  if (!g_init_ok || !g_allow_fused_update) return false;
+  if (g.epi != EPI_PLAIN || g.a_sm != 1 || g.b_sn != 1 || g.c_dt != DT_F32 || g.a_dt != g.b_dt) return false;
+  if (g.M <= 0 || g.N <= 0 || g.K <= 0) return false;
+  const bool tf32 = (g.a_dt == DT_F32);
+  const int esz = tf32 ? 4 : 2;
+  if ((reinterpret_cast<uintptr_t>(g.A) & 15u) || (reinterpret_cast<uintptr_t>(g.B) & 15u)) return false;
+  if ((g.a_sk * esz) % 16 != 0 || (g.b_sk * esz) % 16 != 0) return false;
+  if ((reinterpret_cast<uintptr_t>(g.C) & 15u) || (g.ldc & 3)) return false;
+  const bool throughput = g.off_critical_path != 0;
+  const int split = (g_allow_splitk && !throughput) ? pick_split(g.M, g.N, g.K, tf32) : 1;
+  return split == 1;
+}
+
 cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s, int* family) {
   if (!g_init_ok) return cudaErrorNotSupported;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return cudaErrorNotSupported;
@@ -1317,6 +1486,9 @@ cudaError_t launch_gemm_tc(const GemmDesc& g, int* dev_status, cudaStream_t s, i
   e.C = g.C; e.ldc = g.ldc; e.c_dt = g.c_dt; e.c_round = g.c_round; e.epi = g.epi; e.relu = g.relu;
   e.bias = g.bias; e.mask = g.mask; e.ldmask = g.ldmask;
   e.loss = g.loss; e.loss.enabled = fuse_loss ? 1 : 0;
+  e.upd = g.upd;
+  if (e.upd.enabled && (split > 1 || !a_mn || !b_mn || g.epi != EPI_PLAIN || g.c_dt != DT_F32))
+    return cudaErrorInvalidValue;                           // the caller asks gemm_tc_can_fuse_update first
 
   if (family) *family = pairs ? FAM_TC_PAIR : (split > 1 ? FAM_TC_SPLITK : FAM_TC_SINGLE);
   if (pairs) {

@@ -46,7 +46,7 @@ struct LayerInfo {
   int64_t w_off, b_off;  // element offsets into the flat ranges
 };
 
-enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_UNUSED4, K_UPDATE, K_COPY, K_COUNT };   // values are part of the ABI
+enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_WGRAD_UPDATE, K_UPDATE, K_COPY, K_COUNT };   // values are part of the ABI
 
 int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 
@@ -63,6 +63,7 @@ struct seg_handle {
   bool use_tc = false;
   bool force_tc = false;           // SEG_GEMM_TCGEN05: a product the tensor-core path cannot take is an error
   uint64_t family_launches[FAM_COUNT] = {0, 0, 0, 0};
+  uint64_t fused_updates = 0;      // weight-gradient products that also applied the optimizer update
   int act_dt = DT_F32, act_round = RND_NONE, op_dt = DT_F32, op_round = RND_NONE;
   std::vector<int> widths;
   std::vector<LayerInfo> layers;
@@ -95,6 +96,7 @@ struct seg_handle {
     cudaGraphExec_t exec = nullptr;
     uint64_t kernels = 0, kernels_peer = 0;
     uint64_t family[FAM_COUNT] = {0, 0, 0, 0}, family_peer[FAM_COUNT] = {0, 0, 0, 0};
+    uint64_t fused = 0;
     seg_handle* peer = nullptr;
     cudaGraphNode_t stage_node = nullptr;
     cudaKernelNodeParams stage_params{};
@@ -110,6 +112,8 @@ struct seg_handle {
   bool graphs_enabled = true;
   bool fuse_loss = true;           // take the intermediate-label loss in the last forward product's epilogue where possible
   bool fork_enabled = true;        // run the gradient and update branches on their own streams
+  bool fuse_update = false;        // SEG_FUSED_UPDATE=1: apply the optimizer inside the weight-gradient product where the
+                                   // kernel can (measured slower than the separate update launch, see gemm_tc.cu)
   float* sil = nullptr;
   bool have_labels = false;
   float* loss_partials = nullptr;
@@ -482,6 +486,8 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
     if (env && env[0] == '1') h->fork_enabled = false;
     env = getenv("SEG_NO_FUSED_LOSS");
     if (env && env[0] == '1') h->fuse_loss = false;
+    env = getenv("SEG_FUSED_UPDATE");
+    if (env && env[0] == '1') h->fuse_update = true;
   }
   if (!h->use_tc) {
     // split-K workspaces of the FFMA path, sized for the products each one serves at max_batch
@@ -654,16 +660,35 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
     w.C = h->grads + Ly.w_off; w.ldc = Ly.ldw; w.c_dt = DT_F32; w.c_round = RND_NONE;
     w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
     w.off_critical_path = l > 0;  // the upper layers' weight gradients run beside the dgrad chain and each other
-    if ((st = run_gemm(h, w, K_WGRAD, ls, nullptr, l)) != SEG_OK) return st;
-    // update of W_l and b_l (adjacent in the flat range) once dgrad(l) no longer reads the old W_l
-    if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
     const int64_t lo = Ly.w_off;
+    // Where the persistent tensor-core kernels run the product, they also apply the optimizer to W_l (extra warps
+    // stream over every stored tile, so the update's HBM traffic runs under the main loop); the launch below then
+    // only has the bias left.  The update overwrites W_l's operand copy, which dgrad(l) reads: the fused product
+    // waits for dgrad(l), the separate update does the same one launch later.
+    const bool fused = h->use_tc && h->fuse_update && h->params_op != nullptr && gemm_tc_can_fuse_update(w);
+    if (fused) {
+      if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
+      FusedUpdate& f = w.upd;
+      f.enabled = 1;
+      f.p = h->params + lo;
+      f.s1 = h->state1 ? h->state1 + lo : nullptr; f.s2 = h->state2 ? h->state2 + lo : nullptr;
+      f.p_op = reinterpret_cast<char*>(h->params_op) + lo * elem_size(h->op_dt);
+      f.op_dt = h->op_dt; f.op_round = h->op_round; f.optimizer = h->optimizer;
+      f.lr = h->lr; f.momentum = h->momentum; f.beta1 = h->beta1; f.beta2 = h->beta2; f.eps = h->eps;
+      f.bc = h->bc_dev;
+    }
+    bool w_on_tc = false;
+    if ((st = run_gemm(h, w, fused ? K_WGRAD_UPDATE : K_WGRAD, ls, &w_on_tc, l)) != SEG_OK) return st;
+    if (fused && !w_on_tc) { h->last_error = "fused update product did not run on the tensor-core path"; return SEG_ERR_STATE; }
+    if (fused) ++h->fused_updates;
+    // update of W_l and b_l (adjacent in the flat range) once dgrad(l) no longer reads the old W_l
+    if (branch && !fused) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
     UpdateArgs u{};
     u.p = h->params + lo; u.g = h->grads + lo;
     u.s1 = h->state1 ? h->state1 + lo : nullptr; u.s2 = h->state2 ? h->state2 + lo : nullptr;
     u.p_op = h->params_op ? (void*)(reinterpret_cast<char*>(h->params_op) + lo * elem_size(h->op_dt)) : nullptr;
     u.op_dt = h->op_dt; u.op_round = h->op_round;
-    u.n = Ly.b_off - lo; u.optimizer = h->optimizer;
+    u.n = fused ? 0 : Ly.b_off - lo; u.optimizer = h->optimizer;
     u.dz = dz_l; u.dz_dt = h->act_dt; u.ld_dz = ld_dz; u.batch = batch; u.n_bias = Ly.out;
     u.bias_off = Ly.b_off - lo; u.g_bias = h->grads + Ly.b_off;
     u.lr = h->lr; u.momentum = h->momentum; u.beta1 = h->beta1; u.beta2 = h->beta2; u.eps = h->eps;
@@ -707,6 +732,7 @@ static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const vo
   SEG_TRY(h, cudaGraphLaunch(g.exec, h->stream), "graph launch");
   h->launches += g.kernels;
   for (int f = 0; f < FAM_COUNT; ++f) h->family_launches[f] += g.family[f];
+  h->fused_updates += g.fused;
   if (g.peer) {
     g.peer->launches += g.kernels_peer;
     for (int f = 0; f < FAM_COUNT; ++f) g.peer->family_launches[f] += g.family_peer[f];
@@ -729,8 +755,10 @@ static seg_status run_step_captured(seg_handle* h, seg_handle::StepGraph& g, seg
   const uint64_t before = h->launches, before_peer = peer ? peer->launches : 0;
   uint64_t fam_before[FAM_COUNT], fam_before_peer[FAM_COUNT] = {0, 0, 0, 0};
   for (int f = 0; f < FAM_COUNT; ++f) { fam_before[f] = h->family_launches[f]; if (peer) fam_before_peer[f] = peer->family_launches[f]; }
+  const uint64_t fused_before = h->fused_updates;
   auto restore_counts = [&] {          // what a capture "launched" has not run: take it off the counters again
     h->launches = before;
+    h->fused_updates = fused_before;
     for (int f = 0; f < FAM_COUNT; ++f) h->family_launches[f] = fam_before[f];
     if (peer) {
       peer->launches = before_peer;
@@ -750,6 +778,7 @@ static seg_status run_step_captured(seg_handle* h, seg_handle::StepGraph& g, seg
   if (st == SEG_OK && e == cudaSuccess && graph != nullptr && adopt_captured_graph(h, g, graph)) {
     g.kernels = h->launches - before;
     for (int f = 0; f < FAM_COUNT; ++f) g.family[f] = h->family_launches[f] - fam_before[f];
+    g.fused = h->fused_updates - fused_before;
     g.peer = peer;
     if (peer) {
       g.kernels_peer = peer->launches - before_peer;
@@ -1133,6 +1162,7 @@ seg_status seg_poll_status(seg_handle* h) {
 seg_status seg_product_launches(const seg_handle* h, uint64_t* counts) {
   if (!h || !counts) return SEG_ERR_INVALID_ARG;
   for (int f = 0; f < FAM_COUNT; ++f) counts[f] = h->family_launches[f];
+  counts[FAM_COUNT] = h->fused_updates;
   return SEG_OK;
 }
 

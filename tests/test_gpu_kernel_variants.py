@@ -4,7 +4,9 @@ kernel or the unsplit kernel on their own, so the tensor-core parity cases are r
 processes with the selection forced through the library's environment switches (read once per
 process, hence the child processes).  The same goes for the intermediate-label loss, which the
 tensor-core path takes inside the last forward product's epilogue: SEG_NO_FUSED_LOSS runs the separate
-loss kernel."""
+loss kernel; and for the optimizer update, which the persistent tensor-core kernels apply inside the
+weight-gradient product when SEG_FUSED_UPDATE asks for it (with SEG_NO_SPLITK every weight gradient runs
+in such a kernel)."""
 import os
 import subprocess
 import sys
@@ -17,7 +19,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.mark.parametrize("env", [{"SEG_PAIR_MIN_TILES": "1"}, {"SEG_NO_SPLITK": "1", "SEG_NO_PAIRS": "1"},
                                  {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}, {"SEG_NO_PDL": "1"},
-                                 {"SEG_NO_FUSED_LOSS": "1"}])
+                                 {"SEG_NO_FUSED_LOSS": "1"}, {"SEG_FUSED_UPDATE": "1"}, {"SEG_FUSED_UPDATE": "1", "SEG_NO_SPLITK": "1"}])
 def test_tensor_core_cases_with_forced_kernel_selection(env):
     child_env = dict(os.environ, **env)
     res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",

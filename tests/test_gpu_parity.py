@@ -264,9 +264,13 @@ def expected_families(widths, batch):
     if os.environ.get("SEG_NO_SPLITK") == "1" and os.environ.get("SEG_NO_PAIRS") == "1":
         must.add("tc_single")
     if os.environ.get("SEG_PAIR_MIN_TILES") == "1" and os.environ.get("SEG_NO_PAIRS") != "1":
-        # pairs from one 256 x 256 tile on: any product with M, N, K >= 256 that is not split over K
-        if batch >= 256 and min(widths) >= 256 and os.environ.get("SEG_NO_SPLITK") == "1":
+        # pairs from one 256 x 256 tile on: the products of the 1024-512-512 case are too short to be split over K
+        if batch >= 1024 and min(widths) >= 512:
             must.add("tc_pair")
+    if os.environ.get("SEG_FUSED_UPDATE") != "1":
+        never.add("fused_update")
+    elif os.environ.get("SEG_NO_SPLITK") == "1":
+        must.add("fused_update")                      # every weight gradient runs in a persistent kernel
     return must, never
 
 
@@ -287,7 +291,7 @@ def test_single_step_tensor_core_backend(widths, final, precision, optimizer, ba
     # which kernels ran: every product of both steps on tensor cores, in the family the switches allow
     fam = gpu.product_launches()
     n_products = 2 * (3 * len(widths) - 4)            # per step: L forward, L weight-gradient, L - 1 dgrad products
-    assert sum(fam.values()) == n_products, fam
+    assert sum(fam[f] for f in ("tc_single", "tc_splitk", "tc_pair", "ffma")) == n_products, fam
     must, never = expected_families(widths, batch)
     assert all(fam[f] == 0 for f in never), (fam, never)
     assert all(fam[f] > 0 for f in must), (fam, must)
