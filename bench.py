@@ -645,6 +645,10 @@ def main():
                     help="further workloads summarised in the same line ('' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--samples", type=int, default=0, help="size of the resident data set (0: the workload's own)")
+    ap.add_argument("--quick", action="store_true",
+                    help="warm-up and one timed region only (no end-to-end leg, breakdown, CPU leg or other workloads): "
+                         "the command profilers are pointed at")
+    ap.add_argument("--segment", type=int, default=-1, help="with --quick: run this segment only")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = wl.WORKLOADS[args.workload]
@@ -686,6 +690,18 @@ def main():
         dist.barrier()
     peaks = load_peaks()
     torch.cuda.set_device(local_rank)
+    if args.quick:
+        r = Runner(w, local_rank, host_data=False, n_samples=args.samples or min(w.n_samples, 16 * w.batch))
+        r.prepare()
+        r.gen_labels()
+        r.materialise_inputs()
+        which = args.segment if args.segment >= 0 else None
+        r.run_steps(0, args.warmup, which)
+        ms = r.timed(args.warmup, args.steps, which)
+        print(json.dumps({"quick": True, "workload": w.name, "segment": which, "steps": args.steps,
+                          "ms_per_step": ms / args.steps, "product_launches": r.families()}))
+        r.close()
+        return
     res = measure(w, args.steps, args.warmup, peaks, device_index=local_rank, full=True,
                   n_samples=args.samples or None, extras=not w.concurrent)
     ms_total = res["ms_per_step"] * args.steps
