@@ -38,6 +38,8 @@
  *                         tensor-core kernel runs it (default: a launch of its own, which measured faster)
  *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
  *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
+ *   SEG_NO_STAGED_EPILOGUE=1  persistent product kernels store their output with per-lane stores (default: through
+ *                         shared memory and bulk tensor stores)
  *   SEG_PAIR_MIN_TILES=n  use CTA pairs exactly when a product has n or more tiles of 256 x 256
  *                         (default: a cost model of the main loop chooses)
  *   SEG_DEBUG=1           report on stderr when a step could not be captured into a graph

@@ -116,7 +116,7 @@ def bits_equal(a, b):
 # the band is 5 % of the activation tolerance around zero, i.e. 1e-3 (bf16) / 1e-4 (TF32) of the largest
 # pre-activation, so for a layer whose pre-activations spread over their range the expected share is of
 # that order; ten times that is the ceiling.  fp32 comparisons take nothing from the CUDA path.
-TIE_CEILING = {"fp32": 0.0, "tf32": 1e-3, "bf16": 1e-2}
+TIE_CEILING = {"fp32": 0.0, "tf32": 1e-3, "bf16": 1e-2}      # measured: up to 3.5e-4 / 4.6e-3
 # Units per layer whose decision may actually differ from the oracle's own: a share of the layer, at least 2.
 TIE_FLIPS = {"tf32": 2e-5, "bf16": 2e-4}
 TIE_FLIPS_MIN = 2
@@ -124,9 +124,9 @@ TIE_FLIPS_MIN = 2
 # accumulation, no operand rounding): the figures stated for those paths, 2e-2 (bf16) and 2e-3 (TF32).
 PLAIN_TOL = {"tf32": 2e-3, "bf16": 2e-2}
 # Share of units within the observed activation deviation of zero in the plain-oracle comparison.
-PLAIN_TIE_CEILING = {"tf32": 0.02, "bf16": 0.1}
+PLAIN_TIE_CEILING = {"tf32": 0.005, "bf16": 0.05}       # measured: up to 2.1e-3 / 2.4e-2
 # Adam: smallest share of a tensor's elements that must be in the well-conditioned set (compared at tol).
-ADAM_WELL_FLOOR = 0.02
+ADAM_WELL_FLOOR = 0.4        # measured: 0.58 to 1.0 over all Adam cases
 
 
 def compare_step(gpu, ora, x, cls, precision, tol, check_state=True, ora_plain=None, report=None, tie_scale=1.0):
