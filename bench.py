@@ -36,12 +36,16 @@ from paper_2403_11204_b200 import workloads as wl
 
 L2_BYTES = 126 * 1024 * 1024
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of product kernels, from the ncu captures
-# summarised under profiles/ (the file named beside each figure).  Workloads without a capture of their dominant
-# kind report null.
-NCU_TRAFFIC_BYTES = {("paper_shaped", "fwd_gemm"): (2.621e6, "profiles/gemm_traffic_paper_shaped.md"),
-                     ("paper_shaped", "dgrad_gemm"): (2.953e6, "profiles/gemm_traffic_paper_shaped.md"),
-                     ("paper_shaped", "wgrad_gemm"): (1.326e6, "profiles/gemm_traffic_paper_shaped.md")}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum), mean over the launches of a kind in one step, from
+# the ncu captures summarised under profiles/ (the file named beside each figure).  Workloads without a capture of
+# their dominant kind report null.
+NCU_TRAFFIC_BYTES = {("gemm_large", "fwd_gemm"): (467.6e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "dgrad_gemm"): (597.3e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "wgrad_gemm"): (439.9e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "update"): (1052.8e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("paper_shaped", "fwd_gemm"): (2.623e+06, "profiles/gemm_traffic_paper_shaped.md"),
+                     ("paper_shaped", "dgrad_gemm"): (2.959e+06, "profiles/gemm_traffic_paper_shaped.md"),
+                     ("paper_shaped", "wgrad_gemm"): (1.339e+06, "profiles/gemm_traffic_paper_shaped.md")}
 
 # Rows per oracle step in the CPU legs (full layer widths always): the oracle converts and rounds every weight
 # matrix at each use, so a step of the largest segments costs seconds whatever the batch.
@@ -451,7 +455,8 @@ def kernel_breakdown(r, steps, first, peaks):
     else:
         achieved = v["bytes"] / (v["ms"] * 1e-3) / 1e9
         roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0] if traffic else None,
+                "traffic_source": traffic[1] if traffic else None,
                 "peak_source": f"{peaks['source']}: copy bandwidth", "timing": timing,
                 "launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(v["launches"], 1)}
     return kernels, roof
@@ -757,6 +762,19 @@ def main():
         if extra in res:
             line[extra] = res[extra]
     line["peaks"] = peaks
+    # last, so that it survives a record that keeps only the end of the line: every workload in one compact object
+    def brief(ms, step, segs):
+        return {"ms": round(ms, 4), "sum_frac": round(step["roofline_frac"], 3), "tensor_frac": round(step["tensor_only_frac"], 3),
+                "seg_ms": [round(s_["ms_per_step"], 4) for s_ in segs], "seg_sum_frac": [round(s_["roofline_frac"], 3) for s_ in segs],
+                "seg_tensor_frac": [round(s_["tensor_only_frac"], 3) for s_ in segs]}
+    summary = {w.name: brief(line["ms_per_step"], res["step"], res["segments"])}
+    for name, o in others.items():
+        if "error" not in o:
+            summary[name] = brief(o["ms_per_step"], o["step"], o["segments"])
+    line["summary"] = {"what": "per workload: ms per step; roofline time (product FLOPs at the measured tensor peak + update and loss "
+                               "bytes at the measured copy bandwidth) over step time; product FLOPs over step time over that tensor "
+                               "peak; the same per segment",
+                       **summary}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
