@@ -1074,7 +1074,7 @@ constexpr int PAIR_HALF_N = PAIR_TILE_N / 2;
 constexpr int PAIR_B_BYTES = PAIR_HALF_N * TILE_ROW_BYTES;            // 16 KiB: this CTA's half of B
 constexpr int PAIR_STAGE_BYTES = A_TILE_BYTES + PAIR_B_BYTES;         // 32 KiB per CTA per k-block
 constexpr int PAIR_STAGES = 6;             // without output staging (the fused-update variant)
-constexpr int PAIR_STAGES_STAGED = 5;      // with it: ring + staging stay within the same 192 KiB
+constexpr int PAIR_STAGES_STAGED = 5;      // with it: ring + staging stay within the same 192 KiB (measured: 4 stages +2 %, 3 stages +9 % step time)
 constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + SMEM_EXTRA;   // upper bound of both layouts
 
 template <bool TF32, bool A_MN, bool B_MN, bool FUSED = false>

@@ -60,3 +60,21 @@ def test_class_distributions():
     assert x.dtype == np.float32 and 0.0 <= x.min() and x.max() < 1.0
     b = wl.to_bf16_bits(x)
     assert np.max(np.abs(wl.from_bf16_bits(b) - x)) <= 2 ** -8
+
+
+def test_step_fractions_follow_the_roofline_sum():
+    """roofline time = product FLOPs at the tensor peak + update and loss bytes at the copy bandwidth; the step's fraction
+    is that over the measured time, the tensor-only one counts the products alone."""
+    peaks = {"hbm_gbs": 6000.0, "bf16_tflops": 1500.0, "bf16_tflops_sustained": 1200.0, "source": "test"}
+    work = {"gemm_flops": 3.0e12, "update_bytes": 3.0e9, "loss_bytes": 0.0}
+    f = bench.step_fractions(work, 4.0, "bf16", peaks)            # 2 ms of products + 0.5 ms of update in a 4 ms step
+    assert f["roofline_ms"] == pytest.approx(2.5)
+    assert f["roofline_frac"] == pytest.approx(0.625)
+    assert f["gemm_tflops"] == pytest.approx(750.0)
+    assert f["tensor_only_frac"] == pytest.approx(0.5)
+    assert f["tensor_only_frac_of_sustained_matmul"] == pytest.approx(0.625)
+
+
+def test_cpu_sample_rows_never_exceed_the_batch():
+    for name, w in wl.WORKLOADS.items():
+        assert 1 <= min(w.batch, bench.CPU_SAMPLE_BATCH.get(name, w.batch)) <= w.batch

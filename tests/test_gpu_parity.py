@@ -432,3 +432,41 @@ def test_two_segments_hand_off_through_the_library_copy():
         assert np.max(np.abs(got.cpu().numpy() - want) / np.abs(want)) < 1e-3
     for s_ in segs:
         s_.close()
+
+
+def test_handles_created_and_used_from_two_threads():
+    """Different handles may be created and used from different threads at the same time (the library's one-time set-up
+    and per-device caches are synchronised): two threads each create a tensor-core segment on a stream of their own and
+    run the same three steps; both must end with the bits a single-threaded run gives."""
+    import threading
+    import torch
+    from paper_2403_11204_b200.binding import Segment
+    w = wl.WORKLOADS["tiny"]
+    widths, batch = [256, 384, 128], 192
+    x, cls = batch_arrays(w, batch, widths[0], precision="bf16")
+    xt, ct = to_device(x, cls, "bf16")
+
+    def run(out, use_own_stream):
+        st = torch.cuda.Stream() if use_own_stream else None
+        seg = Segment(widths, 47, False, precision="bf16", optimizer="momentum", lr=0.01, max_batch=batch, stream=st)
+        seg.gen_labels(wl.LABEL_SEED, "normal")
+        loss = torch.zeros(3, device="cuda")
+        for i in range(3):
+            seg.train_step(xt, ct, loss[i:i + 1])
+        seg.poll()
+        W, b = seg.params(0)
+        out.append((loss.cpu().numpy(), W.cpu().numpy(), b.cpu().numpy()))
+        seg.close()
+
+    ref = []
+    run(ref, False)
+    results = [[], []]
+    threads = [threading.Thread(target=run, args=(results[i], True)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(120)
+    for r in results:
+        assert len(r) == 1, "a thread did not finish"
+        for a, b in zip(r[0], ref[0]):
+            assert bits_equal(a, b)
