@@ -49,10 +49,11 @@ struct LossFuse {
 };
 
 // The optimizer update of a layer's weights applied inside its weight-gradient product (tensor-core
-// persistent kernels only): extra warps of every CTA stream over each output tile once the epilogue
-// warps have stored it, so that the update's HBM traffic runs under the main loop of the following
-// tiles instead of after the product.  All pointers address the layer's weight tensor, laid out as
-// the product's C: element (m, n) at base + m * ldc + n.
+// persistent kernels only, opt-in: it measured slower than the separate update launch): extra warps
+// of every CTA stream over each output tile once the epilogue warps have stored it, so that the
+// update's HBM traffic runs under the main loop of the following tiles instead of after the product.
+// All pointers address the layer's weight tensor, laid out as the product's C: element (m, n) at
+// base + m * ldc + n.
 struct FusedUpdate {
   int enabled;              // 0: plain product
   float* p;                 // fp32 master weights

@@ -32,6 +32,18 @@
 // the tensor pipe.  The even CTA issues the MMAs for the pair; TMA loads of both CTAs complete on
 // the even CTA's "full" barrier; one commit frees the stage in both CTAs.
 //
+// The persistent kernels (one CTA or a CTA pair per tile) number their tiles in groups of tile rows
+// sized so that the operand panels a wave of tiles shares stay in L2 (tile_coords, pick_group_m),
+// and store their output through shared memory: each epilogue warp writes its 32 rows x 64 bytes into
+// a staging buffer with the 64-byte swizzle and a bulk tensor store writes the box, clipped to the
+// matrix (epilogue_store_staged).  Ring plus staging stay within 192 KiB: a larger footprint per CTA
+// measured 3-5 % slower over a whole training step although every product alone got faster.
+//
+// An optional variant of both persistent kernels applies the optimizer update inside the
+// weight-gradient product (eight extra warps stream the update of every stored tile).  It measured
+// slower than the separate update launch - the operand loads of the main loop already use most of
+// what L2 delivers to an SM - and is off unless SEG_FUSED_UPDATE=1.
+//
 // Every wait on an mbarrier is bounded: after about two seconds the waiting thread raises an abort
 // flag, records DEV_TIMEOUT in the status word and all roles leave their loops; TMEM is released
 // before the CTA exits.

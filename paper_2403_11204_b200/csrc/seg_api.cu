@@ -661,10 +661,10 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
     w.M = Ly.out; w.N = Ly.in; w.K = batch; w.epi = EPI_PLAIN;
     w.off_critical_path = l > 0;  // the upper layers' weight gradients run beside the dgrad chain and each other
     const int64_t lo = Ly.w_off;
-    // Where the persistent tensor-core kernels run the product, they also apply the optimizer to W_l (extra warps
-    // stream over every stored tile, so the update's HBM traffic runs under the main loop); the launch below then
-    // only has the bias left.  The update overwrites W_l's operand copy, which dgrad(l) reads: the fused product
-    // waits for dgrad(l), the separate update does the same one launch later.
+    // Opt-in (SEG_FUSED_UPDATE=1; measured slower): where the persistent tensor-core kernels run the product, they also
+    // apply the optimizer to W_l (extra warps stream over every stored tile); the launch below then only has the bias
+    // left.  The update overwrites W_l's operand copy, which dgrad(l) reads: the fused product waits for dgrad(l), the
+    // separate update does the same one launch later.
     const bool fused = h->use_tc && h->fuse_update && h->params_op != nullptr && gemm_tc_can_fuse_update(w);
     if (fused) {
       if (branch) SEG_TRY(h, cudaStreamWaitEvent(ls, h->ev_dz[l - 1], 0), "stream wait");
