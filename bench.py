@@ -767,13 +767,13 @@ def main():
         return {"ms": round(ms, 4), "sum_frac": round(step["roofline_frac"], 3), "tensor_frac": round(step["tensor_only_frac"], 3),
                 "seg_ms": [round(s_["ms_per_step"], 4) for s_ in segs], "seg_sum_frac": [round(s_["roofline_frac"], 3) for s_ in segs],
                 "seg_tensor_frac": [round(s_["tensor_only_frac"], 3) for s_ in segs]}
-    summary = {w.name: brief(line["ms_per_step"], res["step"], res["segments"])}
-    for name, o in others.items():
-        if "error" not in o:
-            summary[name] = brief(o["ms_per_step"], o["step"], o["segments"])
-    line["summary"] = {"what": "per workload: ms per step; roofline time (product FLOPs at the measured tensor peak + update and loss "
-                               "bytes at the measured copy bandwidth) over step time; product FLOPs over step time over that tensor "
-                               "peak; the same per segment",
+    summary = {}
+    for name in reversed(list(others)):                 # the headline workload last, the largest others next to it
+        if "error" not in others[name]:
+            summary[name] = brief(others[name]["ms_per_step"], others[name]["step"], others[name]["segments"])
+    summary[w.name] = brief(line["ms_per_step"], res["step"], res["segments"])
+    line["summary"] = {"what": "ms per step; sum_frac = (product FLOPs / tensor peak + update and loss bytes / copy bandwidth) / step time; "
+                               "tensor_frac = product FLOPs / step time / tensor peak; seg_* per segment",
                        **summary}
     print(json.dumps(line))
     if world > 1:

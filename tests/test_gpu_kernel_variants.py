@@ -6,7 +6,7 @@ process, hence the child processes).  The same goes for the intermediate-label l
 tensor-core path takes inside the last forward product's epilogue: SEG_NO_FUSED_LOSS runs the separate
 loss kernel; and for the optimizer update, which the persistent tensor-core kernels apply inside the
 weight-gradient product when SEG_FUSED_UPDATE asks for it (with SEG_NO_SPLITK every weight gradient runs
-in such a kernel); and for the output path of the persistent kernels, staged through shared memory and written by
+in such a kernel, with SEG_PAIR_MIN_TILES=1 the larger ones in the CTA-pair kernel); and for the output path of the persistent kernels, staged through shared memory and written by
 bulk tensor stores by default, per-lane stores with SEG_NO_STAGED_EPILOGUE."""
 import os
 import subprocess
@@ -20,7 +20,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.mark.parametrize("env", [{"SEG_PAIR_MIN_TILES": "1"}, {"SEG_NO_SPLITK": "1", "SEG_NO_PAIRS": "1"},
                                  {"SEG_NO_GRAPH": "1"}, {"SEG_NO_FORK": "1"}, {"SEG_NO_PDL": "1"},
-                                 {"SEG_NO_FUSED_LOSS": "1"}, {"SEG_FUSED_UPDATE": "1"}, {"SEG_FUSED_UPDATE": "1", "SEG_NO_SPLITK": "1"},
+                                 {"SEG_NO_FUSED_LOSS": "1"}, {"SEG_FUSED_UPDATE": "1"},
+                                 {"SEG_FUSED_UPDATE": "1", "SEG_NO_SPLITK": "1", "SEG_PAIR_MIN_TILES": "1"},
                                  {"SEG_NO_STAGED_EPILOGUE": "1"}, {"SEG_NO_STAGED_EPILOGUE": "1", "SEG_PAIR_MIN_TILES": "1"}])
 def test_tensor_core_cases_with_forced_kernel_selection(env):
     child_env = dict(os.environ, **env)
