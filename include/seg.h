@@ -36,6 +36,8 @@
  *                         the last forward product's epilogue where the tensor-core path can take it)
  *   SEG_FUSED_UPDATE=1    apply the optimizer update inside the weight-gradient product where a persistent
  *                         tensor-core kernel runs it (default: a launch of its own, which measured faster)
+ *   SEG_NO_SMALL_FUSED=1  run a small fp32 segment (at most 4 layers of at most 128 units, 1024 inputs) launch by launch
+ *                         (default: its whole step in two launches, see small_step.cu)
  *   SEG_NO_SPLITK=1       never use the cluster split-K product kernel
  *   SEG_NO_PAIRS=1        never use the CTA-pair product kernel
  *   SEG_NO_STAGED_EPILOGUE=1  persistent product kernels store their output with per-lane stores (default: through
@@ -252,7 +254,8 @@ SEG_API seg_status seg_launch_count(const seg_handle* h, uint64_t* launches);
  *   [0] tensor-core, one CTA per tile      [1] tensor-core, K split over a cluster
  *   [2] tensor-core, CTA pair per tile     [3] FFMA
  *   [4] of [0] and [2]: weight-gradient products that also applied the optimizer update
- * Tests use it to show which kernels actually ran.                                           */
+ * The two launches of a small fp32 segment's step (kinds 7 and 4 of seg_profile_get) count as two FFMA
+ * launches and one of [4].  Tests use it to show which kernels actually ran.                                           */
 SEG_API seg_status seg_product_launches(const seg_handle* h, uint64_t* counts);
 
 /* Synchronises the handle's stream and returns SEG_ERR_DEVICE_TIMEOUT if any kernel of
@@ -293,7 +296,9 @@ SEG_API seg_status seg_timer_elapsed_ms(seg_handle* h, float* ms);
  * since profiling was enabled; kinds: 0 forward product, 1 dgrad product, 2 wgrad
  * product, 3 loss, 4 wgrad product that also applies the optimizer update to the weights,
  * 5 optimizer update as a launch of its own (forms the bias gradient too; after a kind-4
- * product it has only the bias left), 6 copies / staging.  count and
+ * product it has only the bias left), 6 copies / staging, 7 the first launch of a small
+ * fp32 segment's two-launch step (staging, forward, loss and dgrad chain; its second launch,
+ * all weight and bias gradients with the update, counts as kind 4).  count and
  * total_ms are host pointers.                                                            */
 SEG_API seg_status seg_profile_enable(seg_handle* h, int32_t on);
 SEG_API seg_status seg_profile_get(seg_handle* h, int32_t kind, uint64_t* count, float* total_ms);

@@ -21,7 +21,8 @@ OPTIMIZERS = {"sgd": SEG_SGD, "momentum": SEG_SGD_MOMENTUM, "adam": SEG_ADAM}
 LABEL_DISTS = {"uniform_kappa": SEG_LABEL_UNIFORM_KAPPA, "normal": SEG_LABEL_NORMAL}
 BACKENDS = {"auto": SEG_GEMM_AUTO, "simt": SEG_GEMM_SIMT, "tcgen05": SEG_GEMM_TCGEN05}
 # kind numbers of seg_profile_get
-KERNEL_KINDS = {0: "fwd_gemm", 1: "dgrad_gemm", 2: "wgrad_gemm", 3: "loss", 4: "wgrad_update_gemm", 5: "update", 6: "copy"}
+KERNEL_KINDS = {0: "fwd_gemm", 1: "dgrad_gemm", 2: "wgrad_gemm", 3: "loss", 4: "wgrad_update_gemm", 5: "update", 6: "copy",
+                7: "fwd_loss_dgrad"}
 # order of the counters seg_product_launches returns (the last one counts a subset of tc_single + tc_pair)
 PRODUCT_FAMILIES = ("tc_single", "tc_splitk", "tc_pair", "ffma", "fused_update")
 

@@ -7,7 +7,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsegtrain.so")
-SOURCES = ["seg_api.cu", "rng.cu", "elementwise.cu", "gemm_simt.cu", "gemm_tc.cu"]
+SOURCES = ["seg_api.cu", "rng.cu", "elementwise.cu", "gemm_simt.cu", "small_step.cu", "gemm_tc.cu"]
 
 
 def _nvcc():

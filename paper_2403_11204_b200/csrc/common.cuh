@@ -227,4 +227,86 @@ __device__ __forceinline__ void store_from_float(void* p, int dt, int64_t i, flo
   else reinterpret_cast<float*>(p)[i] = v;
 }
 
+// ---- whole step of a small fp32 segment in two launches ---------------------------------------------
+// A segment of at most kSmallMaxLayers layers, none wider than kSmallMaxWidth, fed kSmallMaxInput features at
+// most (Section 3: 784-80-60 and 60-60-60-47) is latency-bound when every product, the loss and every update
+// is a launch of its own.  The first kernel carries a slice of the batch through staging, all forward
+// products, the loss and the dgrad chain; the second forms every layer's weight and bias gradient and
+// applies the optimizer.  Description of one step for both (all pointers device, fp32):
+constexpr int kSmallMaxLayers = 4, kSmallMaxWidth = 128, kSmallMaxInput = 1024;
+struct SmallStep {
+  int n_layers, batch, n_classes, is_final, last_relu, optimizer;
+  int widths[kSmallMaxLayers + 1];
+  int64_t ldw[kSmallMaxLayers], w_off[kSmallMaxLayers], b_off[kSmallMaxLayers];   // element offsets into the flat ranges
+  int64_t ld_act[kSmallMaxLayers + 1];
+  float* params; float* grads; float* s1; float* s2;
+  float* act[kSmallMaxLayers + 1];     // act[0]: the staged input
+  float* dz[kSmallMaxLayers];
+  const float* sil;
+  int32_t* cls_stage;
+  float* loss_partials; unsigned int* loss_counter; float** loss_dst;
+  unsigned long long* t; float* bc;
+  int* dev_status;
+  float lr, momentum, beta1, beta2, eps;
+  float* wg_scratch; unsigned int* wg_counters; int wg_slots;   // partial 64 x 64 tiles of the weight-gradient kernel
+};
+bool small_step_supported(int n_layers, const int* widths);   // the shape limits above
+bool small_step_batch_ok(int batch);                          // one loss partial per CTA: bounded by loss_max_partials()
+int small_step_wgrad_slots(int n_layers, const int* widths);  // partial tiles (and counters) the second kernel may use
+cudaError_t launch_small_fwd_bwd(const SmallStep& p, const float* x, const int32_t* cls, const float* gather,
+                                 float* loss_to, cudaStream_t s);
+cudaError_t launch_small_wgrad_update(const SmallStep& p, cudaStream_t s);
+
+// ---- reductions -------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+// Sum over the block in a fixed order (deterministic for a fixed launch shape); valid in warp 0.
+__device__ inline float block_sum(float v, float* smem /* >= 32 floats */) {
+  v = warp_sum(v);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane == 0) smem[warp] = v;
+  __syncthreads();
+  float total = 0.f;
+  if (warp == 0) {
+    const int n_warps = (blockDim.x + 31) >> 5;
+    total = lane < n_warps ? smem[lane] : 0.f;
+    total = warp_sum(total);
+  }
+  return total;
+}
+// Writes this block's partial; the last block to finish adds all partials in index order and
+// writes scale * total to loss_out, or, when loss_dst is not null, to the address stored in
+// *loss_dst.  The counter is left at zero for the next launch.
+__device__ inline void finish_loss(float block_total, float* partials, unsigned int* counter,
+                            float* loss_out, float* const* loss_dst, float scale, float* smem) {
+  __shared__ bool is_last;
+  if (threadIdx.x == 0) {
+    partials[blockIdx.x] = block_total;
+    __threadfence();
+    const unsigned int done = atomicAdd(counter, 1u);
+    is_last = (done == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    float v = 0.f;
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += blockDim.x) v += __ldcg(partials + i);
+    const float total = block_sum(v, smem);
+    if (threadIdx.x == 0) {
+      if (loss_dst) loss_out = *loss_dst;
+      if (loss_out) *loss_out = total * scale;
+      *counter = 0u;
+    }
+  }
+}
+
 }  // namespace segk

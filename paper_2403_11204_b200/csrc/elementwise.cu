@@ -13,59 +13,6 @@ namespace {
 constexpr int kLossThreads = 256;
 constexpr int kMaxLossBlocks = 1024;
 
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-  return v;
-}
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-  return v;
-}
-
-// Sum over the block in a fixed order (deterministic for a fixed launch shape).
-__device__ float block_sum(float v, float* smem /* >= 32 floats */) {
-  v = warp_sum(v);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  __syncthreads();
-  if (lane == 0) smem[warp] = v;
-  __syncthreads();
-  float total = 0.f;
-  if (warp == 0) {
-    const int n_warps = (blockDim.x + 31) >> 5;
-    total = lane < n_warps ? smem[lane] : 0.f;
-    total = warp_sum(total);
-  }
-  return total;  // valid in warp 0
-}
-
-// Writes this block's partial; the last block to finish adds all partials in index order and
-// writes scale * total to loss_out, or, when loss_dst is not null, to the address stored in
-// *loss_dst.  The counter is left at zero for the next launch.
-__device__ void finish_loss(float block_total, float* partials, unsigned int* counter,
-                            float* loss_out, float* const* loss_dst, float scale, float* smem) {
-  __shared__ bool is_last;
-  if (threadIdx.x == 0) {
-    partials[blockIdx.x] = block_total;
-    __threadfence();
-    const unsigned int done = atomicAdd(counter, 1u);
-    is_last = (done == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (is_last) {
-    __threadfence();
-    float v = 0.f;
-    for (int i = threadIdx.x; i < (int)gridDim.x; i += blockDim.x) v += __ldcg(partials + i);
-    const float total = block_sum(v, smem);
-    if (threadIdx.x == 0) {
-      if (loss_dst) loss_out = *loss_dst;
-      if (loss_out) *loss_out = total * scale;
-      *counter = 0u;
-    }
-  }
-}
-
 // Non-final segment: target of sample b is row cls[b] of the label matrix (gathered here, never
 // materialised per sample);  loss = mean (a - t)^2,  dZ = 2 (a - t) / (B N_P) * [a > 0].
 // A thread handles VEC consecutive columns of one row per pass (VEC = 8: 16-byte accesses for bf16,
@@ -143,8 +90,10 @@ mse_loss_kernel(const TOut* __restrict__ out, int64_t ld_out, const int32_t* __r
 }
 
 // Final segment: one warp per sample;  p = softmax(z) with the row maximum subtracted,
-// loss = -mean log p[cls],  dZ = (p - onehot) / B.
-template <typename TDz>
+// loss = -mean log p[cls],  dZ = (p - onehot) / B.  Rows of up to 32 * CE_REGS classes are read once and kept
+// in registers (lane i holds classes i, i + 32, ...); wider rows are read three times.
+constexpr int CE_REGS = 32;
+template <typename TDz, bool IN_REGS>
 __global__ void __launch_bounds__(kLossThreads)
 softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* __restrict__ cls,
                   int n_classes, int batch, int relu_mask, TDz* __restrict__ dz, int dz_round,
@@ -160,23 +109,56 @@ softmax_ce_kernel(const float* __restrict__ logits, int64_t ld, const int32_t* _
   for (int b = blockIdx.x * warps_per_block + (threadIdx.x >> 5); b < batch;
        b += gridDim.x * warps_per_block) {
     const float* z = logits + (int64_t)b * ld;
-    float mx = -INFINITY;
-    for (int i = lane; i < n_classes; i += 32) mx = fmaxf(mx, z[i]);
-    mx = warp_max(mx);
-    float se = 0.f;
-    for (int i = lane; i < n_classes; i += 32) se += expf(z[i] - mx);
-    se = warp_sum(se);
-    const int c = __ldg(cls + b);
-    const float inv_se = 1.0f / se;
-    for (int i = lane; i < n_classes; i += 32) {
-      const float zi = z[i];
-      float g = (expf(zi - mx) * inv_se - (i == c ? 1.f : 0.f)) * inv_b;
-      if (relu_mask && !(zi > 0.f)) g = 0.f;
-      g = apply_round(g, dz_round);
-      if constexpr (sizeof(TDz) == 2) dz[(int64_t)b * ld_dz + i] = __float2bfloat16_rn(g);
-      else dz[(int64_t)b * ld_dz + i] = g;
+    const int c = min(max(__ldg(cls + b), 0), n_classes - 1);
+    if constexpr (IN_REGS) {
+      float v[CE_REGS];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < CE_REGS; ++j) {
+        const int i = lane + 32 * j;
+        v[j] = i < n_classes ? z[i] : -INFINITY;
+        mx = fmaxf(mx, v[j]);
+      }
+      mx = warp_max(mx);
+      float se = 0.f;
+#pragma unroll
+      for (int j = 0; j < CE_REGS; ++j)
+        if (lane + 32 * j < n_classes) se += expf(v[j] - mx);
+      se = warp_sum(se);
+      const float inv_se = 1.0f / se;
+      float zc = 0.f;
+#pragma unroll
+      for (int j = 0; j < CE_REGS; ++j) {
+        const int i = lane + 32 * j;
+        if (i < n_classes) {
+          float g = (expf(v[j] - mx) * inv_se - (i == c ? 1.f : 0.f)) * inv_b;
+          if (relu_mask && !(v[j] > 0.f)) g = 0.f;
+          g = apply_round(g, dz_round);
+          if constexpr (sizeof(TDz) == 2) dz[(int64_t)b * ld_dz + i] = __float2bfloat16_rn(g);
+          else dz[(int64_t)b * ld_dz + i] = g;
+          if (i == c) zc = v[j];
+        }
+      }
+      zc = warp_sum(zc);                       // exactly one lane holds the class's logit, the others 0
+      if (lane == 0) acc += logf(se) - (zc - mx);
+    } else {
+      float mx = -INFINITY;
+      for (int i = lane; i < n_classes; i += 32) mx = fmaxf(mx, z[i]);
+      mx = warp_max(mx);
+      float se = 0.f;
+      for (int i = lane; i < n_classes; i += 32) se += expf(z[i] - mx);
+      se = warp_sum(se);
+      const float inv_se = 1.0f / se;
+      for (int i = lane; i < n_classes; i += 32) {
+        const float zi = z[i];
+        float g = (expf(zi - mx) * inv_se - (i == c ? 1.f : 0.f)) * inv_b;
+        if (relu_mask && !(zi > 0.f)) g = 0.f;
+        g = apply_round(g, dz_round);
+        if constexpr (sizeof(TDz) == 2) dz[(int64_t)b * ld_dz + i] = __float2bfloat16_rn(g);
+        else dz[(int64_t)b * ld_dz + i] = g;
+      }
+      if (lane == 0) acc += logf(se) - (z[c] - mx);
     }
-    if (lane == 0) acc += logf(se) - (z[c] - mx);
   }
   const float bt = block_sum(acc, red);
   finish_loss(bt, partials, counter, loss_out, loss_dst, inv_b, red);
@@ -418,15 +400,16 @@ cudaError_t launch_softmax_ce_loss(const float* logits, int64_t ld_logits, const
   float* const loss_out = nullptr;
   const int warps = kLossThreads / 32;
   const int grid = grid_for(batch, warps, kMaxLossBlocks);
+  const bool in_regs = n_classes <= 32 * CE_REGS;
+#define SEGK_CE(TD, R)                                                                                         \
+  launch_k(softmax_ce_kernel<TD, R>, dim3(grid), dim3(kLossThreads), 0, s, logits, ld_logits, cls, n_classes, \
+           batch, relu_mask, (TD*)dz, dz_round, ld_dz, partials, counter, loss_out, loss_dst)
   if (dz_dt == DT_BF16) {
-    launch_k(softmax_ce_kernel<__nv_bfloat16>, dim3(grid), dim3(kLossThreads), 0, s, 
-        logits, ld_logits, cls, n_classes, batch, relu_mask, (__nv_bfloat16*)dz, dz_round, ld_dz,
-        partials, counter, loss_out, loss_dst);
+    if (in_regs) SEGK_CE(__nv_bfloat16, true); else SEGK_CE(__nv_bfloat16, false);
   } else {
-    launch_k(softmax_ce_kernel<float>, dim3(grid), dim3(kLossThreads), 0, s, logits, ld_logits, cls, n_classes,
-                                                          batch, relu_mask, (float*)dz, dz_round,
-                                                          ld_dz, partials, counter, loss_out, loss_dst);
+    if (in_regs) SEGK_CE(float, true); else SEGK_CE(float, false);
   }
+#undef SEGK_CE
   return cudaGetLastError();
 }
 

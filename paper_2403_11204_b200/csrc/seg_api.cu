@@ -46,9 +46,15 @@ struct LayerInfo {
   int64_t w_off, b_off;  // element offsets into the flat ranges
 };
 
-enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_WGRAD_UPDATE, K_UPDATE, K_COPY, K_COUNT };   // values are part of the ABI
+enum Kind { K_FWD = 0, K_DGRAD, K_WGRAD, K_LOSS, K_WGRAD_UPDATE, K_UPDATE, K_COPY, K_FWD_BWD, K_COUNT };   // values are part of the ABI
 
 int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+// Position of the caller-supplied pointers in the parameter list of the kernel that takes them in: the input
+// staging kernel (see elementwise.cu), or the first kernel of a small segment's two-launch step.
+struct StageArgs { int count, x, cls, gather, loss; };
+constexpr StageArgs kStageInputsArgs = {19, 3, 9, 14, 15};
+constexpr StageArgs kSmallStepArgs = {5, 1, 2, 3, 4};
 
 }  // namespace
 
@@ -99,12 +105,14 @@ struct seg_handle {
     uint64_t fused = 0;
     seg_handle* peer = nullptr;
     cudaGraphNode_t stage_node = nullptr;
+    StageArgs stage_idx{};
     cudaKernelNodeParams stage_params{};
     std::vector<void*> stage_args;
     const void* cur_x = nullptr; const int32_t* cur_cls = nullptr; float* cur_loss = nullptr;   // now in the exec
     const float* cur_gather = nullptr;
   };
   cudaGraphNode_t cap_stage_node = nullptr;   // filled while capturing
+  StageArgs cap_stage_idx{};
   bool capturing = false;
   std::map<int, StepGraph> graphs; // by batch size
   std::map<std::pair<uint64_t, int>, StepGraph> recovery_graphs;   // by (right segment's uid, batch size)
@@ -112,6 +120,8 @@ struct seg_handle {
   bool graphs_enabled = true;
   bool fuse_loss = true;           // take the intermediate-label loss in the last forward product's epilogue where possible
   bool fork_enabled = true;        // run the gradient and update branches on their own streams
+  bool small_fused = false;        // small fp32 segment: the whole step runs as two launches (SEG_NO_SMALL_FUSED=1: off)
+  SmallStep small{};               // its description, filled by seg_create (batch is set per step)
   bool fuse_update = false;        // SEG_FUSED_UPDATE=1: apply the optimizer inside the weight-gradient product where the
                                    // kernel can (measured slower than the separate update launch, see gemm_tc.cu)
   float* sil = nullptr;
@@ -514,6 +524,32 @@ seg_status seg_create(const seg_config* cfg, seg_handle** out) {
   if ((st = dev_alloc(h, &h->loss_partials, loss_max_partials(), true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->loss_counter, 1, true)) != SEG_OK) return bail(st);
   if ((st = dev_alloc(h, &h->dev_status, 1, true)) != SEG_OK) return bail(st);
+  {
+    const char* env = getenv("SEG_NO_SMALL_FUSED");
+    h->small_fused = h->precision == SEG_FP32 && !(env && env[0] == '1') &&
+                     small_step_supported(h->n_layers, h->widths.data());
+  }
+  if (h->small_fused) {
+    SmallStep& p = h->small;
+    p.n_layers = h->n_layers; p.n_classes = h->n_classes; p.is_final = h->is_final ? 1 : 0;
+    p.last_relu = h->last_relu ? 1 : 0; p.optimizer = h->optimizer;
+    for (int l = 0; l <= h->n_layers; ++l) {
+      p.widths[l] = h->widths[l]; p.ld_act[l] = h->ld_act[l];
+      p.act[l] = reinterpret_cast<float*>(l == 0 ? h->x_stage : h->act[l]);
+    }
+    for (int l = 0; l < h->n_layers; ++l) {
+      p.ldw[l] = h->layers[l].ldw; p.w_off[l] = h->layers[l].w_off; p.b_off[l] = h->layers[l].b_off;
+      p.dz[l] = reinterpret_cast<float*>(h->dzbuf[l]);
+    }
+    p.params = h->params; p.grads = h->grads; p.s1 = h->state1; p.s2 = h->state2;
+    p.sil = h->sil; p.cls_stage = h->cls_stage;
+    p.loss_partials = h->loss_partials; p.loss_counter = h->loss_counter; p.loss_dst = h->loss_dst;
+    p.t = h->step_dev; p.bc = h->bc_dev; p.dev_status = h->dev_status;
+    p.lr = h->lr; p.momentum = h->momentum; p.beta1 = h->beta1; p.beta2 = h->beta2; p.eps = h->eps;
+    p.wg_slots = small_step_wgrad_slots(h->n_layers, h->widths.data());
+    if ((st = dev_alloc(h, &p.wg_scratch, (size_t)p.wg_slots * kSimtTileFloats, false)) != SEG_OK) return bail(st);
+    if ((st = dev_alloc(h, &p.wg_counters, p.wg_slots, true)) != SEG_OK) return bail(st);
+  }
   if (cudaEventCreate(&h->ev_start) != cudaSuccess || cudaEventCreate(&h->ev_stop) != cudaSuccess)
     return bail(SEG_ERR_CUDA);
 
@@ -608,6 +644,26 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
   cudaStream_t mainst = h->stream;
   seg_status st;
   float* loss_to = loss_out ? loss_out : h->loss_slot;
+  if (h->small_fused && small_step_batch_ok(batch)) {
+    // small fp32 segment: staging, forward, loss and the dgrad chain in one launch, every weight and bias
+    // gradient with its update in a second
+    SmallStep p = h->small;
+    p.batch = batch;
+    {
+      Launch lf(h, K_FWD_BWD);
+      SEG_TRY(h, launch_small_fwd_bwd(p, reinterpret_cast<const float*>(x), cls, gather, loss_to, mainst),
+              "small-segment forward/backward launch");
+    }
+    if (h->capturing) { h->cap_stage_node = last_captured_node(h); h->cap_stage_idx = kSmallStepArgs; }
+    {
+      Launch lw(h, K_WGRAD_UPDATE);
+      SEG_TRY(h, launch_small_wgrad_update(p, mainst), "small-segment weight-gradient/update launch");
+    }
+    h->family_launches[FAM_SIMT] += 2;
+    ++h->fused_updates;
+    h->last_batch = batch;
+    return SEG_OK;
+  }
   {
     // fixed staging buffers: rounds x in TF32 mode, pads the pitch, keeps every later pointer constant;
     // the same launch advances the device-side step counter and Adam's bias corrections and records
@@ -617,7 +673,7 @@ static seg_status enqueue_step(seg_handle* h, int batch, bool forked, const void
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
                                    gather, loss_to, h->loss_dst, h->n_classes, h->dev_status, mainst), "input staging");
   }
-  if (h->capturing) h->cap_stage_node = last_captured_node(h);
+  if (h->capturing) { h->cap_stage_node = last_captured_node(h); h->cap_stage_idx = kStageInputsArgs; }
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch, h->cls_stage, h->loss_dst)) != SEG_OK) return st;
   return enqueue_backward(h, batch, forked);
 }
@@ -704,14 +760,12 @@ static seg_status enqueue_backward(seg_handle* h, int batch, bool forked) {
   return SEG_OK;
 }
 
-// Index of the caller-supplied pointers in the kernels' parameter lists (see elementwise.cu).
-static const int kStageArgCount = 19, kStageArgX = 3, kStageArgCls = 9, kStageArgGather = 14, kStageArgLoss = 15;
-
 static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGraph_t graph) {
   if (!h->cap_stage_node) return false;
   g.stage_node = h->cap_stage_node;
+  g.stage_idx = h->cap_stage_idx;
   if (cudaGraphKernelNodeGetParams(g.stage_node, &g.stage_params) != cudaSuccess) return false;
-  g.stage_args.assign(g.stage_params.kernelParams, g.stage_params.kernelParams + kStageArgCount);
+  g.stage_args.assign(g.stage_params.kernelParams, g.stage_params.kernelParams + g.stage_idx.count);
   if (cudaGraphInstantiate(&g.exec, graph, 0) != cudaSuccess) { g.exec = nullptr; return false; }
   g.graph = graph;                      // kept alive: the parameter blocks above belong to it
   return true;
@@ -720,10 +774,10 @@ static bool adopt_captured_graph(seg_handle* h, seg_handle::StepGraph& g, cudaGr
 static seg_status replay_graph(seg_handle* h, seg_handle::StepGraph& g, const void* x, const int32_t* cls,
                                float* loss_to, const float* gather) {
   if (x != g.cur_x || cls != g.cur_cls || gather != g.cur_gather || loss_to != g.cur_loss) {
-    g.stage_args[kStageArgX] = (void*)&x;
-    g.stage_args[kStageArgCls] = (void*)&cls;
-    g.stage_args[kStageArgGather] = (void*)&gather;
-    g.stage_args[kStageArgLoss] = (void*)&loss_to;
+    g.stage_args[g.stage_idx.x] = (void*)&x;
+    g.stage_args[g.stage_idx.cls] = (void*)&cls;
+    g.stage_args[g.stage_idx.gather] = (void*)&gather;
+    g.stage_args[g.stage_idx.loss] = (void*)&loss_to;
     cudaKernelNodeParams sp = g.stage_params;
     sp.kernelParams = g.stage_args.data();
     SEG_TRY(h, cudaGraphExecKernelNodeSetParams(g.exec, g.stage_node, &sp), "graph parameter update");
@@ -848,7 +902,7 @@ static seg_status enqueue_recovery(seg_handle* h, seg_handle* r, int batch, bool
                                    h->act_round, h->cls_stage, cls, h->step_dev, h->bc_dev, h->beta1, h->beta2,
                                    nullptr, loss_to, h->loss_dst, h->n_classes, h->dev_status, s), "input staging");
   }
-  if (h->capturing) h->cap_stage_node = last_captured_node(h);
+  if (h->capturing) { h->cap_stage_node = last_captured_node(h); h->cap_stage_idx = kStageInputsArgs; }
   if ((st = forward_layers(h, h->x_stage, h->ld_act[0], batch)) != SEG_OK) return st;
   // the joined network's loss: the right segment's softmax cross-entropy on the class labels
   if ((st = forward_layers(r, h->act[Ll], h->ld_act[Ll], batch, h->cls_stage, h->loss_dst)) != SEG_OK) return st;

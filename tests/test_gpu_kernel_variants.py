@@ -7,7 +7,9 @@ tensor-core path takes inside the last forward product's epilogue: SEG_NO_FUSED_
 loss kernel; and for the optimizer update, which the persistent tensor-core kernels apply inside the
 weight-gradient product when SEG_FUSED_UPDATE asks for it (with SEG_NO_SPLITK every weight gradient runs
 in such a kernel, with SEG_PAIR_MIN_TILES=1 the larger ones in the CTA-pair kernel); and for the output path of the persistent kernels, staged through shared memory and written by
-bulk tensor stores by default, per-lane stores with SEG_NO_STAGED_EPILOGUE."""
+bulk tensor stores by default, per-lane stores with SEG_NO_STAGED_EPILOGUE.  Small fp32 segments run
+their whole step in two launches; SEG_NO_SMALL_FUSED sends them through the launch-by-launch path, so
+the fp32 cases run once more that way."""
 import os
 import subprocess
 import sys
@@ -27,4 +29,12 @@ def test_tensor_core_cases_with_forced_kernel_selection(env):
     child_env = dict(os.environ, **env)
     res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",
                           "-k", "tensor_core"], cwd=ROOT, env=child_env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-1000:]
+
+
+def test_fp32_cases_launch_by_launch():
+    child_env = dict(os.environ, SEG_NO_SMALL_FUSED="1")
+    res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",
+                          "-k", "fp32 or tiny or reproducible or replayed or class_index"], cwd=ROOT, env=child_env,
+                         capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-1000:]

@@ -55,6 +55,13 @@ SMALL = [
     ([60, 60, 60, 47], True, "fp32", "momentum", 141),
     ([100, 72, 40], False, "fp32", "adam", 33),
     ([40, 24, 47], True, "fp32", "adam", 1),
+    # wider than the two-launch step of small segments takes: the FFMA products, loss and update kernels
+    ([200, 160, 96], False, "fp32", "adam", 50),
+    ([96, 160, 47], True, "fp32", "momentum", 50),
+    # four layers; a batch large enough for the 16-row slices, with a ragged last slice
+    ([33, 128, 7, 128, 12], False, "fp32", "momentum", 77),
+    ([60, 60, 47], True, "fp32", "sgd", 2405),
+    ([1024, 47], True, "fp32", "adam", 9),
 ]
 
 
@@ -69,6 +76,34 @@ def test_single_step_fp32(widths, final, precision, optimizer, batch):
         sync_from_oracle(gpu, ora)
     compare_step(gpu, ora, x2, cls2, precision, TOL[precision])      # second step: optimizer state in play
     gpu.close()
+
+
+def test_small_fp32_segment_steps_in_two_launches():
+    """A small fp32 segment (the paper's 784-80-60 and 60-60-60-47) runs its whole step as two launches:
+    the launch counter grows by two per step, eager, captured and replayed alike, both count as FFMA and one as a
+    weight-gradient product that applied the update; a wider segment goes launch by launch."""
+    import os
+    if os.environ.get("SEG_NO_SMALL_FUSED") == "1":
+        pytest.skip("the two-launch step is switched off in this process")
+    w = wl.WORKLOADS["paper_net"]
+    for widths, final, small in (([784, 80, 60], False, True), ([60, 60, 60, 47], True, True),
+                                 ([784, 160, 60], False, False)):
+        gpu, _ = make_pair(widths, 47, final, "fp32", "momentum", 0.01, 141)
+        x, cls = batch_arrays(w, 141, widths[0])
+        xt, ct = to_device(x, cls, "fp32")
+        counts = []
+        for _ in range(4):
+            before = gpu.launch_count()
+            gpu.train_step(xt, ct)
+            counts.append(gpu.launch_count() - before)
+        gpu.poll()
+        fam = gpu.product_launches()
+        if small:
+            assert counts == [2, 2, 2, 2], counts
+            assert (fam["ffma"], fam["fused_update"]) == (8, 4), fam
+        else:
+            assert min(counts) > 6 and fam["fused_update"] == 0, (counts, fam)
+        gpu.close()
 
 
 @pytest.mark.parametrize("label_dist", ["uniform_kappa", "normal"])
