@@ -278,15 +278,23 @@ stage_inputs_kernel(void* dst, int dt, int64_t ld_dst, const void* src, int64_t 
   pdl_wait();
   pdl_trigger();
   const int64_t total = (int64_t)rows * cols;
-  const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  const int64_t n_threads = (int64_t)gridDim.x * blockDim.x;
-  if (tid == 0 && loss_dst != nullptr) *loss_dst = loss_out;   // where this step's loss kernel writes the loss
-  if (tid == 0 && t != nullptr) {           // step counter and Adam bias corrections of this step
-    const unsigned long long step = *t + 1ull;
-    *t = step;
-    bc[0] = (float)(1.0 - pow((double)beta1, (double)step));
-    bc[1] = (float)(1.0 - pow((double)beta2, (double)step));
+  // The last block only keeps the books (the two double-precision powers take longer than a copying thread's
+  // share of a small batch; in a block of their own they run beside the copy instead of in front of it).
+  const int copy_blocks = (int)gridDim.x - 1;
+  if ((int)blockIdx.x == copy_blocks) {
+    if (threadIdx.x == 0) {
+      if (loss_dst != nullptr) *loss_dst = loss_out;   // where this step's loss kernel writes the loss
+      if (t != nullptr) {                              // step counter and Adam bias corrections of this step
+        const unsigned long long step = *t + 1ull;
+        *t = step;
+        bc[0] = (float)(1.0 - pow((double)beta1, (double)step));
+        bc[1] = (float)(1.0 - pow((double)beta2, (double)step));
+      }
+    }
+    return;
   }
+  const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const int64_t n_threads = (int64_t)copy_blocks * blockDim.x;
   const int esz = dt == DT_BF16 ? 2 : 4;
   const bool dst_wide = ((cols * esz) & 15) == 0 && ((ld_dst * esz) & 15) == 0 &&
                         (reinterpret_cast<uintptr_t>(dst) & 15u) == 0;
@@ -441,7 +449,7 @@ cudaError_t launch_stage_inputs(void* dst, int dt, int64_t ld_dst, const void* s
                                 const float* gather_src, float* loss_out, float** loss_dst,
                                 int n_classes, int* dev_status, cudaStream_t s) {
   const int esz = dt == DT_BF16 ? 2 : 4;
-  const int grid = grid_for((int64_t)rows * cols * esz / 16, 256, 148 * 8);   // one 16-byte group per thread and pass
+  const int grid = grid_for((int64_t)rows * cols * esz / 16, 256, 148 * 8) + 1;   // one 16-byte group per thread and pass; + the bookkeeping block
   launch_k(stage_inputs_kernel, dim3(grid), dim3(256), 0, s, dst, dt, ld_dst, src, ld_src, rows, cols, round, cls_dst, cls_src, t, bc,
                                            beta1, beta2, gather_src, loss_out, loss_dst, n_classes, dev_status);
   return cudaGetLastError();

@@ -244,16 +244,17 @@ struct SmemLayout {
 // global-memory latency is off the critical path.
 struct EpiSide { uint32_t w[32]; };
 
+template <int NV = 32>
 __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide& s, int row, bool row_ok,
                                                   int col0, int n_total) {
-  const int n_valid = min(32, n_total - col0);
+  const int n_valid = min(NV, n_total - col0);
   if (n_valid <= 0) return;
   const bool whole = (n_valid & 7) == 0;
   if (e.epi == EPI_BIAS_ACT) {
     const float* brow = e.bias + col0;
     if (whole && ((reinterpret_cast<uintptr_t>(brow) & 15u) == 0)) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 4) {
+      for (int j = 0; j < NV; j += 4) {
         if (j < n_valid) {
           const uint4 b = __ldg(reinterpret_cast<const uint4*>(brow + j));
           s.w[j] = b.x; s.w[j + 1] = b.y; s.w[j + 2] = b.z; s.w[j + 3] = b.w;
@@ -261,14 +262,14 @@ __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < n_valid) s.w[j] = __float_as_uint(__ldg(brow + j));
+      for (int j = 0; j < NV; ++j) if (j < n_valid) s.w[j] = __float_as_uint(__ldg(brow + j));
     }
   } else if (e.epi == EPI_MASK && row_ok) {
     if (e.c_dt == DT_BF16) {
       const unsigned short* mrow = reinterpret_cast<const unsigned short*>(e.mask) + (int64_t)row * e.ldmask + col0;
       if (whole && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0)) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 8) {
+        for (int j = 0; j < NV; j += 8) {
           if (j < n_valid) {
             const uint4 q = __ldg(reinterpret_cast<const uint4*>(mrow + j));
             s.w[j / 2] = q.x; s.w[j / 2 + 1] = q.y; s.w[j / 2 + 2] = q.z; s.w[j / 2 + 3] = q.w;
@@ -276,7 +277,7 @@ __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
+        for (int j = 0; j < NV; j += 2) {
           uint32_t lo = 0u, hi = 0u;
           if (j < n_valid) lo = __ldg(mrow + j);
           if (j + 1 < n_valid) hi = __ldg(mrow + j + 1);
@@ -287,7 +288,7 @@ __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide
       const float* mrow = reinterpret_cast<const float*>(e.mask) + (int64_t)row * e.ldmask + col0;
       if (whole && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0)) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
+        for (int j = 0; j < NV; j += 4) {
           if (j < n_valid) {
             const uint4 m = __ldg(reinterpret_cast<const uint4*>(mrow + j));
             s.w[j] = m.x; s.w[j + 1] = m.y; s.w[j + 2] = m.z; s.w[j + 3] = m.w;
@@ -295,7 +296,7 @@ __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) if (j < n_valid) s.w[j] = __float_as_uint(__ldg(mrow + j));
+        for (int j = 0; j < NV; ++j) if (j < n_valid) s.w[j] = __float_as_uint(__ldg(mrow + j));
       }
     }
   }
@@ -305,46 +306,48 @@ __device__ __forceinline__ void epilogue_prefetch(const EpilogueArgs& e, EpiSide
 // Columns are stored in groups of 8 with 16-byte accesses when the group count is whole and the
 // row segment is 16-byte aligned (every lane touches its own row, so wide accesses are what keeps
 // the number of memory wavefronts down); ragged or unaligned segments fall back to scalar stores.
-__device__ __forceinline__ void epilogue_values(const EpilogueArgs& e, float (&v)[32], const EpiSide& s, int col0,
+template <int NV>
+__device__ __forceinline__ void epilogue_values(const EpilogueArgs& e, float (&v)[NV], const EpiSide& s, int col0,
                                                 int n_total) {
-  const int n_valid = min(32, n_total - col0);
+  const int n_valid = min(NV, n_total - col0);
   if (e.epi == EPI_BIAS_ACT) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) if (j < n_valid) v[j] += __uint_as_float(s.w[j]);
+    for (int j = 0; j < NV; ++j) if (j < n_valid) v[j] += __uint_as_float(s.w[j]);
     if (e.relu) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+      for (int j = 0; j < NV; ++j) v[j] = fmaxf(v[j], 0.f);
     }
   } else if (e.epi == EPI_MASK) {
     if (e.c_dt == DT_BF16) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
+      for (int j = 0; j < NV; ++j) {
         // a bf16 is positive iff its sign bit is clear and it is not zero
         const uint32_t bits = (s.w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
         if (j < n_valid && !(bits != 0u && bits < 0x8000u)) v[j] = 0.f;
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
+      for (int j = 0; j < NV; ++j)
         if (j < n_valid && !(__uint_as_float(s.w[j]) > 0.f)) v[j] = 0.f;
     }
   }
   if (e.c_round == RND_TF32) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = round_tf32_rne(v[j]);
+    for (int j = 0; j < NV; ++j) v[j] = round_tf32_rne(v[j]);
   }
 }
 
 // Stores up to 32 consecutive columns of one row into a [rows][ld] matrix of dtype dt.
-__device__ __forceinline__ void store_row_segment(void* base, int dt, int64_t ld, const float (&v)[32], int row,
+template <int NV>
+__device__ __forceinline__ void store_row_segment(void* base, int dt, int64_t ld, const float (&v)[NV], int row,
                                                   int col0, int n_total) {
-  const int n_valid = min(32, n_total - col0);
+  const int n_valid = min(NV, n_total - col0);
   const bool whole = (n_valid & 7) == 0;
   if (dt == DT_BF16) {
     __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(base) + (int64_t)row * ld + col0;
     if (whole && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 8) {
+      for (int j = 0; j < NV; j += 8) {
         if (j < n_valid) {
           uint4 q;
           __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]);
@@ -358,23 +361,24 @@ __device__ __forceinline__ void store_row_segment(void* base, int dt, int64_t ld
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < n_valid) crow[j] = __float2bfloat16_rn(v[j]);
+      for (int j = 0; j < NV; ++j) if (j < n_valid) crow[j] = __float2bfloat16_rn(v[j]);
     }
   } else {
     float* crow = reinterpret_cast<float*>(base) + (int64_t)row * ld + col0;
     if (whole && ((reinterpret_cast<uintptr_t>(crow) & 15u) == 0)) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 4) {
+      for (int j = 0; j < NV; j += 4) {
         if (j < n_valid) *reinterpret_cast<float4*>(crow + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < n_valid) crow[j] = v[j];
+      for (int j = 0; j < NV; ++j) if (j < n_valid) crow[j] = v[j];
     }
   }
 }
 
-__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[32], const EpiSide& s, int row,
+template <int NV>
+__device__ __forceinline__ void epilogue_store(const EpilogueArgs& e, float (&v)[NV], const EpiSide& s, int row,
                                                int col0, int n_total) {
   epilogue_values(e, v, s, col0, n_total);
   store_row_segment(e.C, e.c_dt, e.ldc, v, row, col0, n_total);
@@ -438,13 +442,14 @@ __device__ __forceinline__ float warp_sum_f(float v) {
 
 // Targets of n_cols (<= 32) consecutive columns of one row: row cls[row] of the label matrix, whose
 // pitch is n_p.  Fetched ahead of the accumulator like the other side inputs.
+template <int NV = 32>
 __device__ __forceinline__ void loss_prefetch_target(const LossFuse& l, EpiSide& t, int row, bool row_ok, int col0,
                                                      int n_cols, int n_p) {
   if (n_cols <= 0 || !row_ok) return;
   const float* trow = l.sil + (int64_t)__ldg(l.cls + row) * n_p + col0;
   if (((n_cols & 3) == 0) && ((reinterpret_cast<uintptr_t>(trow) & 15u) == 0)) {
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < NV; j += 4) {
       if (j < n_cols) {
         const uint4 q = __ldg(reinterpret_cast<const uint4*>(trow + j));
         t.w[j] = q.x; t.w[j + 1] = q.y; t.w[j + 2] = q.z; t.w[j + 3] = q.w;
@@ -452,20 +457,21 @@ __device__ __forceinline__ void loss_prefetch_target(const LossFuse& l, EpiSide&
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) if (j < n_cols) t.w[j] = __float_as_uint(__ldg(trow + j));
+    for (int j = 0; j < NV; ++j) if (j < n_cols) t.w[j] = __float_as_uint(__ldg(trow + j));
   }
 }
 
 // Mean-squared-error part of the epilogue for columns [col0, n_end): stores the output, then
 // dZ = gscale (a - t) [a > 0], and adds (a - t)^2 to the thread's loss sum; a is the output as it
 // is stored (after rounding to the storage type).
-__device__ __forceinline__ void epilogue_store_mse(const EpilogueArgs& e, float (&v)[32], const EpiSide& s,
+template <int NV>
+__device__ __forceinline__ void epilogue_store_mse(const EpilogueArgs& e, float (&v)[NV], const EpiSide& s,
                                                    const EpiSide& t, int row, int col0, int n_end, float& lacc) {
   epilogue_values(e, v, s, col0, n_end);
   store_row_segment(e.C, e.c_dt, e.ldc, v, row, col0, n_end);
-  const int n_valid = min(32, n_end - col0);
+  const int n_valid = min(NV, n_end - col0);
 #pragma unroll
-  for (int j = 0; j < 32; ++j) {
+  for (int j = 0; j < NV; ++j) {
     if (j < n_valid) {
       const float a = (e.c_dt == DT_BF16) ? round_bf16_rne(v[j]) : v[j];
       const float d = a - __uint_as_float(t.w[j]);
@@ -678,13 +684,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
+      int fills = 0;                     // stages filled so far, counted up to the ring's depth: the first pass waits for nothing
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
         int m_idx, n_idx;
         tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
         const int m0 = m_idx * BLOCK_M, n0 = n_idx * BLOCK_N;
         for (int kb = 0; kb < num_k; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
+          if (fills < STAGES) ++fills;
+          else if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
           mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::STAGE_BYTES);
           const uint32_t a_dst = smem_u32(smem_a + stage * A_TILE_BYTES);
           const uint32_t b_dst = smem_u32(smem_b + stage * L::B_TILE_BYTES);
@@ -838,10 +846,13 @@ constexpr int SPLITK_RECV_BYTES = 8 * (SPLITK_BLOCK_N / 8) * BLOCK_M * 4;       
 constexpr int SPLITK_SMEM = SPLITK_STAGES * SPLITK_STAGE_BYTES + 2 * SPLITK_RECV_BYTES + SMEM_EXTRA;   // + send buffer
 
 // One 128 x 64 output tile per cluster; CTA r of the cluster contracts k-blocks [r*kpc, (r+1)*kpc).
-template <bool TF32, bool A_MN, bool B_MN, bool LOSS = false>
+template <bool TF32, bool A_MN, bool B_MN, int SPLIT, bool LOSS = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                      int M, int N, int K, int split, EpilogueArgs epi, int* dev_status) {
+                      int M, int N, int K, EpilogueArgs epi, int* dev_status) {
+  constexpr int split = SPLIT;                             // CTAs per cluster
+  constexpr int W = SPLITK_BLOCK_N / SPLIT;                // columns of the tile each CTA owns after the exchange
+  static_assert(W == 32 || W == 16 || W == 8, "slice width");
   constexpr int BLOCK_N = SPLITK_BLOCK_N;
   constexpr int STAGES = SPLITK_STAGES;
   constexpr int B_TILE_BYTES = BLOCK_N * TILE_ROW_BYTES;
@@ -891,9 +902,7 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   cluster_arrive();                   // "my barriers are initialised"; the matching wait sits in front of the
   tc_fence_after();                   // first remote access (the slice exchange), off the main loop's path
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();
-  pdl_trigger();
-
+  // tile and k-range of this CTA: index arithmetic only, done while the previous kernel drains
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   const int tile = blockIdx.x / split;
   const int m0 = (tile % tiles_m) * BLOCK_M, n0 = (tile / tiles_m) * BLOCK_N;
@@ -901,15 +910,23 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   const int kpc = (num_k + split - 1) / split;
   const int kb_begin = min(num_k, (int)rank * kpc), kb_end = min(num_k, kb_begin + kpc);
   const int my_k = kb_end - kb_begin;     // may be 0 for the last ranks: they contribute zeros
+  pdl_wait();
+  pdl_trigger();
 
+  // The k-loop of such a small product is bound by how fast one thread can issue the loads (a few hundred cycles
+  // per k-block), so two threads share it: this warp announces the stage's bytes and loads the A tiles, the first
+  // epilogue warp, idle until the accumulator is complete, loads the B tiles.  Both wait for the stage to be
+  // free; bytes of B that land before the announcement only take the barrier's byte count below zero for a while
+  // (the phase cannot complete before the announcing arrival).
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) break;
+        // the first pass over the ring finds every stage free: no wait (a wait that passes at once still costs a
+        // couple of hundred cycles of the issuing thread)
+        if (kb - kb_begin >= STAGES && !mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) break;
         mbar_arrive_expect_tx(full_bar(stage), (uint32_t)SPLITK_STAGE_BYTES);
         const uint32_t a_dst = smem_u32(smem_a + stage * A_TILE_BYTES);
-        const uint32_t b_dst = smem_u32(smem_b + stage * B_TILE_BYTES);
         const int k0 = kb * BLOCK_K;
         if constexpr (A_MN) {
 #pragma unroll
@@ -917,13 +934,6 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             tma_load_2d(a_dst + c * MN_CHUNK_BYTES, &map_a, m0 + c * CHUNK, k0, full_bar(stage));
         } else {
           tma_load_2d(a_dst, &map_a, k0, m0, full_bar(stage));
-        }
-        if constexpr (B_MN) {
-#pragma unroll
-          for (int c = 0; c < BLOCK_N / CHUNK; ++c)
-            tma_load_2d(b_dst + c * MN_CHUNK_BYTES, &map_b, n0 + c * CHUNK, k0, full_bar(stage));
-        } else {
-          tma_load_2d(b_dst, &map_b, k0, n0, full_bar(stage));
         }
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
@@ -962,21 +972,40 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     }
   } else {
     // ---------------- epilogue warps: reduce-scatter across the cluster, then the usual epilogue ------------
+    if (warp == 2 && lane == 0) {                          // first: the B tiles of the main loop (see above)
+      int stage = 0; uint32_t phase = 0;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        // the first pass over the ring finds every stage free: no wait (a wait that passes at once still costs a
+        // couple of hundred cycles of the issuing thread)
+        if (kb - kb_begin >= STAGES && !mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) break;
+        const uint32_t b_dst = smem_u32(smem_b + stage * B_TILE_BYTES);
+        const int k0 = kb * BLOCK_K;
+        if constexpr (B_MN) {
+#pragma unroll
+          for (int c = 0; c < BLOCK_N / CHUNK; ++c)
+            tma_load_2d(b_dst + c * MN_CHUNK_BYTES, &map_b, n0 + c * CHUNK, k0, full_bar(stage));
+        } else {
+          tma_load_2d(b_dst, &map_b, k0, n0, full_bar(stage));
+        }
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+    __syncwarp();
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
     const int row = m0 + row_in_tile;
-    const int w = BLOCK_N / split;                         // columns owned by each CTA: 32, 16 or 8
+    constexpr int w = W;                                   // columns owned by each CTA: 32, 16 or 8
     const int own_col0 = n0 + (int)rank * w;
     EpiSide side, tgt;                                     // side inputs of this CTA's slice, fetched ahead
-    epilogue_prefetch(epi, side, row, row < M, own_col0, min(N, own_col0 + w));
-    if constexpr (LOSS) loss_prefetch_target(epi.loss, tgt, row, row < M, own_col0, min(w, N - own_col0), N);
+    epilogue_prefetch<W>(epi, side, row, row < M, own_col0, min(N, own_col0 + w));
+    if constexpr (LOSS) loss_prefetch_target<W>(epi.loss, tgt, row, row < M, own_col0, min(w, N - own_col0), N);
     float lacc = 0.f;
     bool ok = mbar_wait(acc_bar, 0, abort_flag, dev_status);
     tc_fence_after();
     const uint32_t slice_bytes = (uint32_t)(w * BLOCK_M * 4);
-    float own[32];                                         // this CTA's slice of its own partial (w <= 32 used)
+    float own[W];                                          // this CTA's slice of the tile
 #pragma unroll
-    for (int j = 0; j < 32; ++j) own[j] = 0.f;
+    for (int j = 0; j < W; ++j) own[j] = 0.f;
     if (ok) {
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
@@ -1009,13 +1038,11 @@ gemm_tc_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     }
     if (ok) {
 #pragma unroll
-      for (int cs = 0; cs < 32; ++cs)
-        if (cs < w) own[cs] = send[((int)rank * w + cs) * BLOCK_M + row_in_tile];
+      for (int cs = 0; cs < W; ++cs) own[cs] = send[((int)rank * w + cs) * BLOCK_M + row_in_tile];
       for (int src = 0; src < split; ++src) {
         if ((uint32_t)src == rank) continue;
 #pragma unroll
-        for (int cs = 0; cs < 32; ++cs)
-          if (cs < w) own[cs] += recv[(src * w + cs) * BLOCK_M + row_in_tile];
+        for (int cs = 0; cs < W; ++cs) own[cs] += recv[(src * w + cs) * BLOCK_M + row_in_tile];
       }
       if (row < M && own_col0 < N) {
         if constexpr (LOSS) epilogue_store_mse(epi, own, side, tgt, row, own_col0, min(N, own_col0 + w), lacc);
@@ -1151,6 +1178,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ---------------- TMA producer (both CTAs; completion on the even CTA's barrier) ----------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
+      int fills = 0;                     // as in the single-CTA kernel: no wait on the first pass over the ring
       bool ok = true;
       for (int t = pair; t < n_tiles && ok; t += n_pairs) {
         int m_idx, n_idx;
@@ -1158,7 +1186,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int m0 = m_idx * PAIR_TILE_M + (int)rank * BLOCK_M;
         const int n0 = n_idx * PAIR_TILE_N + (int)rank * PAIR_HALF_N;
         for (int kb = 0; kb < num_k; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
+          if (fills < STAGES) ++fills;
+          else if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) { ok = false; break; }
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(2 * PAIR_STAGE_BYTES));
           const uint32_t fb = map_to_cta(full_bar(stage), 0);
           const uint32_t a_dst = smem_u32(smem_a + stage * A_TILE_BYTES);
@@ -1416,10 +1445,11 @@ cudaError_t launch_majors(bool a_mn, bool b_mn, const CUtensorMap& ma, const CUt
 }
 
 
-template <bool TF32, bool A_MN, bool B_MN, bool LOSS = false>
-cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
-                                  const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
-  auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN, LOSS>;
+template <bool TF32, bool A_MN, bool B_MN, int SPLIT, bool LOSS = false>
+cudaError_t launch_splitk_cluster(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
+                                  const EpilogueArgs& e, int* dev_status, cudaStream_t s) {
+  constexpr int split = SPLIT;
+  auto kern = gemm_tc_splitk_kernel<TF32, A_MN, B_MN, SPLIT, LOSS>;
   static std::atomic<bool> attr_set_dev[kMaxDevices];      // the attribute is per device
   if (cudaError_t err = ensure_dynamic_smem(kern, SPLITK_SMEM, attr_set_dev); err != cudaSuccess) return err;
   const int tiles = ((g.M + BLOCK_M - 1) / BLOCK_M) * ((g.N + SPLITK_BLOCK_N - 1) / SPLITK_BLOCK_N);
@@ -1434,7 +1464,17 @@ cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, 
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = g_use_pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, kern, ma, mb, g.M, g.N, g.K, split, e, dev_status);
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, g.M, g.N, g.K, e, dev_status);
+}
+
+template <bool TF32, bool A_MN, bool B_MN, bool LOSS = false>
+cudaError_t launch_splitk_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmDesc& g,
+                                  const EpilogueArgs& e, int split, int* dev_status, cudaStream_t s) {
+  switch (split) {
+    case 2: return launch_splitk_cluster<TF32, A_MN, B_MN, 2, LOSS>(ma, mb, g, e, dev_status, s);
+    case 4: return launch_splitk_cluster<TF32, A_MN, B_MN, 4, LOSS>(ma, mb, g, e, dev_status, s);
+    default: return cudaErrorNotSupported;                  // pick_split chooses 2 or 4
+  }
 }
 
 template <bool TF32>

@@ -189,8 +189,10 @@ small_fwd_bwd_kernel(const __grid_constant__ SmallStep p, const float* __restric
   if (blockIdx.x == 0 && tid == 0) {
     const unsigned long long step = *p.t + 1ull;
     *p.t = step;
-    p.bc[0] = (float)(1.0 - pow((double)p.beta1, (double)step));
-    p.bc[1] = (float)(1.0 - pow((double)p.beta2, (double)step));
+    if (p.optimizer == SEG_ADAM) {      // the only reader of the bias corrections; two double-precision powers cost over a microsecond
+      p.bc[0] = (float)(1.0 - pow((double)p.beta1, (double)step));
+      p.bc[1] = (float)(1.0 - pow((double)p.beta2, (double)step));
+    }
     *p.loss_dst = loss_to;
   }
   if (tid < R) {
