@@ -39,12 +39,12 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum), mean over the launches of a kind in one step, from
 # the ncu captures summarised under profiles/ (the file named beside each figure).  Workloads without a capture of
 # their dominant kind report null.
-NCU_TRAFFIC_BYTES = {("gemm_large", "fwd_gemm"): (467.6e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("gemm_large", "dgrad_gemm"): (597.3e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("gemm_large", "wgrad_gemm"): (439.9e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("gemm_large", "update"): (1052.8e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("paper_shaped", "fwd_gemm"): (2.623e+06, "profiles/gemm_traffic_paper_shaped.md"),
-                     ("paper_shaped", "dgrad_gemm"): (2.959e+06, "profiles/gemm_traffic_paper_shaped.md"),
+NCU_TRAFFIC_BYTES = {("gemm_large", "fwd_gemm"): (470.2e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "dgrad_gemm"): (598.6e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "wgrad_gemm"): (470.6e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "update"): (1052.9e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("paper_shaped", "fwd_gemm"): (2.613e+06, "profiles/gemm_traffic_paper_shaped.md"),
+                     ("paper_shaped", "dgrad_gemm"): (2.955e+06, "profiles/gemm_traffic_paper_shaped.md"),
                      ("paper_shaped", "wgrad_gemm"): (1.339e+06, "profiles/gemm_traffic_paper_shaped.md")}
 
 # Rows per oracle step in the CPU legs (full layer widths always): the oracle converts and rounds every weight
