@@ -672,13 +672,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();                         // everything above overlapped the previous kernel's tail
-  pdl_trigger();
-
+  // index arithmetic (several integer divisions), the first tile's coordinates included: ahead of the dependency wait
   const int tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
   const int tiles_n = (N + BLOCK_N - 1) / BLOCK_N;
   const int n_tiles = tiles_m * tiles_n;
   const int num_k = (K + BLOCK_K - 1) / BLOCK_K;
+  int first_m = 0, first_n = 0;
+  if ((int)blockIdx.x < n_tiles) tile_coords((int)blockIdx.x, tiles_m, tiles_n, group_m, first_m, first_n);
+  pdl_wait();                         // everything above overlapped the previous kernel's tail
+  pdl_trigger();
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -688,7 +690,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
         int m_idx, n_idx;
-        tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
+        if (t == (int)blockIdx.x) { m_idx = first_m; n_idx = first_n; } else tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
         const int m0 = m_idx * BLOCK_M, n0 = n_idx * BLOCK_N;
         for (int kb = 0; kb < num_k; ++kb) {
           if (fills < STAGES) ++fills;
@@ -762,7 +764,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
       int m_idx, n_idx;
-      tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
+      if (t == (int)blockIdx.x) { m_idx = first_m; n_idx = first_n; } else tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
       const int m0 = m_idx * BLOCK_M, n0 = n_idx * BLOCK_N;
       const int row = m0 + quarter * 32 + lane;
       EpiSide side, side_next;
@@ -802,7 +804,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         needed += 4u;
         if (!tile_stored_wait(tiles_done, needed, abort_flag, dev_status, lane)) break;
         int m_idx, n_idx;
-        tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
+        if (t == (int)blockIdx.x) { m_idx = first_m; n_idx = first_n; } else tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
         const int m0 = m_idx * BLOCK_M, n0 = n_idx * BLOCK_N;
         update_tile<BLOCK_N>(epi.upd, reinterpret_cast<const float*>(epi.C), epi.ldc, m0, n0, M, N, uw, lane,
                              inv_bc1, inv_bc2);
@@ -1165,14 +1167,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   cluster_wait();                     // both CTAs' barriers exist before any cross-CTA signal
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();
-  pdl_trigger();
-
+  // index arithmetic, the first tile's coordinates included: ahead of the dependency wait
   const int tiles_m = (M + PAIR_TILE_M - 1) / PAIR_TILE_M;
   const int tiles_n = (N + PAIR_TILE_N - 1) / PAIR_TILE_N;
   const int n_tiles = tiles_m * tiles_n;
   const int num_k = (K + BLOCK_K - 1) / BLOCK_K;
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  int first_m = 0, first_n = 0;
+  if (pair < n_tiles) tile_coords(pair, tiles_m, tiles_n, group_m, first_m, first_n);
+  pdl_wait();
+  pdl_trigger();
 
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs; completion on the even CTA's barrier) ----------------
@@ -1182,7 +1186,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       bool ok = true;
       for (int t = pair; t < n_tiles && ok; t += n_pairs) {
         int m_idx, n_idx;
-        tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
+        if (t == pair) { m_idx = first_m; n_idx = first_n; } else tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
         const int m0 = m_idx * PAIR_TILE_M + (int)rank * BLOCK_M;
         const int n0 = n_idx * PAIR_TILE_N + (int)rank * PAIR_HALF_N;
         for (int kb = 0; kb < num_k; ++kb) {
@@ -1256,7 +1260,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     bool ok = true;
     for (int t = pair; t < n_tiles && ok; t += n_pairs) {
       int m_idx, n_idx;
-      tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
+      if (t == pair) { m_idx = first_m; n_idx = first_n; } else tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
       const int m0 = m_idx * PAIR_TILE_M + (int)rank * BLOCK_M;
       const int n0 = n_idx * PAIR_TILE_N;
       const int row = m0 + quarter * 32 + lane;
@@ -1297,7 +1301,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         needed += 4u;
         if (!tile_stored_wait(tiles_done, needed, abort_flag, dev_status, lane)) break;
         int m_idx, n_idx;
-        tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
+        if (t == pair) { m_idx = first_m; n_idx = first_n; } else tile_coords(t, tiles_m, tiles_n, group_m, m_idx, n_idx);
         const int m0 = m_idx * PAIR_TILE_M + (int)rank * BLOCK_M;
         const int n0 = n_idx * PAIR_TILE_N;
         update_tile<PAIR_TILE_N>(epi.upd, reinterpret_cast<const float*>(epi.C), epi.ldc, m0, n0, M, N, uw, lane,
