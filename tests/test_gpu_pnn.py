@@ -75,17 +75,19 @@ def test_recovery_step_matches_the_oracle(precision, backend, tol):
     gl.close(); gr.close()
 
 
-@pytest.mark.parametrize("precision,backend,tol", [("fp32", "auto", 1e-4), ("bf16", "tcgen05", 2e-2)])
-def test_fully_separate_variant_label_rows_as_input(precision, backend, tol):
+@pytest.mark.parametrize("precision,backend,tol,hidden", [("fp32", "auto", 1e-4, 200), ("fp32", "auto", 1e-4, 96),
+                                                          ("bf16", "tcgen05", 2e-2, 200)])
+def test_fully_separate_variant_label_rows_as_input(precision, backend, tol, hidden):
     """Section 2, last flowchart: a middle partition trained with the previous cut's labels as input and
-    its own cut's labels as target; the input rows are gathered by class on the device."""
+    its own cut's labels as target; the input rows are gathered by class on the device (by the staging
+    kernel, or, hidden = 96, inside the first launch of a small fp32 segment's two-launch step)."""
     import torch
     from oracle import rng as orng
     from parity_util import compare_step, bits_equal
     w = wl.WORKLOADS["tiny"]
     m, batch = 47, 150
     prev_labels = orng.gen_labels(wl.LABEL_SEED, 0, m, 136, orng.DIST_UNIFORM_KAPPA, 10.0)     # cut 0: 47 x 136
-    gpu, ora = make_pair([136, 200, 72], m, False, precision, "momentum", 0.01, batch, segment_id=1,
+    gpu, ora = make_pair([136, hidden, 72], m, False, precision, "momentum", 0.01, batch, segment_id=1,
                          gemm_backend=backend, label_dist="uniform_kappa")
     cls = wl.class_indices(w, batch)
     sil_t = torch.from_numpy(prev_labels).cuda()
