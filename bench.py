@@ -39,13 +39,13 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum), mean over the launches of a kind in one step, from
 # the ncu captures summarised under profiles/ (the file named beside each figure).  Workloads without a capture of
 # their dominant kind report null.
-NCU_TRAFFIC_BYTES = {("gemm_large", "fwd_gemm"): (470.2e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("gemm_large", "dgrad_gemm"): (598.6e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("gemm_large", "wgrad_gemm"): (470.6e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("gemm_large", "update"): (1052.9e6, "profiles/gemm_traffic_gemm_large.md"),
-                     ("paper_shaped", "fwd_gemm"): (2.613e+06, "profiles/gemm_traffic_paper_shaped.md"),
+NCU_TRAFFIC_BYTES = {("gemm_large", "fwd_gemm"): (469.9e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "dgrad_gemm"): (598.1e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "wgrad_gemm"): (451.6e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("gemm_large", "update"): (1052.2e6, "profiles/gemm_traffic_gemm_large.md"),
+                     ("paper_shaped", "fwd_gemm"): (2.614e+06, "profiles/gemm_traffic_paper_shaped.md"),
                      ("paper_shaped", "dgrad_gemm"): (2.955e+06, "profiles/gemm_traffic_paper_shaped.md"),
-                     ("paper_shaped", "wgrad_gemm"): (1.339e+06, "profiles/gemm_traffic_paper_shaped.md")}
+                     ("paper_shaped", "wgrad_gemm"): (1.340e+06, "profiles/gemm_traffic_paper_shaped.md")}
 
 # Rows per oracle step in the CPU legs (full layer widths always): the oracle converts and rounds every weight
 # matrix at each use, so a step of the largest segments costs seconds whatever the batch.
