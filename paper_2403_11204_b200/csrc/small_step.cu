@@ -7,9 +7,10 @@
 //   1. small_fwd_bwd_kernel gives every CTA a slice of R rows of the batch and carries it through the
 //      whole chain: input staging (class clamp, gather of label rows), all forward products with bias
 //      and ReLU, the loss and dZ of the last layer, and the dgrad chain.  Activations and dZ of the slice
-//      stay in shared memory (stored k-major, so that a thread reads its rows with one 16-byte load);
-//      weights are streamed through a 32-row shared tile.  Every activation and dZ also goes to global
-//      memory, where the second kernel (and seg_get_activation) reads it.
+//      stay in shared memory (stored k-major, so that a thread reads its rows with 16-byte loads); the
+//      weights of all products of the chain arrive as one stream of 64-row tiles through a cp.async ring.
+//      Every activation and dZ also goes to global memory, where the second kernel (and
+//      seg_get_activation) reads it.
 //   2. small_wgrad_update_kernel forms dW_l = dZ_l^T A_{l-1} of all layers in one grid of 64 x 64 tiles,
 //      the batch split over several CTAs per tile; the bias gradient is the column a ones-vector appended
 //      to A_{l-1} yields.  The last CTA of a tile to arrive adds the partial tiles in split order (a fixed
@@ -381,19 +382,32 @@ small_wgrad_update_kernel(SmallStep p, int splits, int k_per_split) {
   const int64_t ld_dz = p.ld_act[l + 1], ld_a = p.ld_act[l];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int k_begin = z * k_per_split, k_end = min(p.batch, k_begin + k_per_split);
-  constexpr int LD = WT * WK / SS_THREADS;
-  float ra[LD], rb[LD];
+  // A k-step of each operand is 32 rows of 64 floats = 512 groups of 4: two per thread.  A group inside the
+  // buffer's pitch is one 16-byte load (rows are 32-byte aligned; what lies between the width and the pitch is
+  // zero, and products with it are never stored); the group of A_{l-1} that holds column `in` (the ones) or
+  // crosses the width is put together element by element.
+  constexpr int LD = WT * WK / 4 / SS_THREADS;
+  float4 ra[LD], rb[LD];
   float acc[4][4] = {};
   auto fetch = [&](int k0) {
 #pragma unroll
     for (int i = 0; i < LD; ++i) {
       const int idx = threadIdx.x + SS_THREADS * i;
-      const int c = idx & (WT - 1), k = k0 + (idx >> 6);
-      ra[i] = 0.f; rb[i] = 0.f;
+      const int c = (idx & 15) * 4, k = k0 + (idx >> 4);
+      ra[i] = make_float4(0.f, 0.f, 0.f, 0.f); rb[i] = ra[i];
       if (k < k_end) {
-        if (m0 + c < out) ra[i] = dz[(int64_t)k * ld_dz + m0 + c];
-        if (n0 + c < in) rb[i] = ap[(int64_t)k * ld_a + n0 + c];
-        else if (n0 + c == in) rb[i] = 1.0f;
+        if (m0 + c + 3 < ld_dz) ra[i] = *reinterpret_cast<const float4*>(dz + (int64_t)k * ld_dz + m0 + c);
+        if (n0 + c + 3 < in) {
+          rb[i] = *reinterpret_cast<const float4*>(ap + (int64_t)k * ld_a + n0 + c);
+        } else {
+          float t[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int cc = n0 + c + j;
+            t[j] = cc < in ? ap[(int64_t)k * ld_a + cc] : (cc == in ? 1.0f : 0.f);
+          }
+          rb[i] = make_float4(t[0], t[1], t[2], t[3]);
+        }
       }
     }
   };
@@ -402,8 +416,8 @@ small_wgrad_update_kernel(SmallStep p, int splits, int k_per_split) {
 #pragma unroll
     for (int i = 0; i < LD; ++i) {
       const int idx = threadIdx.x + SS_THREADS * i;
-      As[idx >> 6][idx & (WT - 1)] = ra[i];
-      Bs[idx >> 6][idx & (WT - 1)] = rb[i];
+      *reinterpret_cast<float4*>(&As[idx >> 4][(idx & 15) * 4]) = ra[i];
+      *reinterpret_cast<float4*>(&Bs[idx >> 4][(idx & 15) * 4]) = rb[i];
     }
     __syncthreads();
     if (k0 + WK < k_end) fetch(k0 + WK);
@@ -457,18 +471,39 @@ small_wgrad_update_kernel(SmallStep p, int splits, int k_per_split) {
   }
   float inv_bc1 = 1.0f, inv_bc2 = 1.0f;
   if constexpr (OPT == SEG_ADAM) { inv_bc1 = 1.0f / __ldg(p.bc); inv_bc2 = 1.0f / __ldg(p.bc + 1); }
-  // this thread's 16 elements: all loads first (they do not depend on one another), then the arithmetic and the stores
+  // this thread's 16 elements (4 rows of 4 consecutive columns): all loads first (they do not depend on one
+  // another), then the arithmetic and the stores.  A row segment that lies wholly inside the weight matrix moves
+  // with 16-byte accesses (rows of W are 32-byte aligned and the segment starts at a multiple of 4 columns); the
+  // ragged segment at the matrix edge, which also carries the bias element, goes element by element.
   int64_t e[4][4];
+  bool wide[4];
   float w[4][4], m[4][4], v[4][4];
+  const int c0 = n0 + tx * 4;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int o = m0 + ty * 4 + i;
+    wide[i] = o < out && c0 + 3 < in;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int c = n0 + tx * 4 + j;
+      const int c = c0 + j;
       e[i][j] = (o >= out || c > in) ? -1 : (c < in ? p.w_off[l] + (int64_t)o * p.ldw[l] + c : p.b_off[l] + o);
       w[i][j] = 0.f; m[i][j] = 0.f; v[i][j] = 0.f;
-      if (e[i][j] >= 0) {
+    }
+    if (wide[i]) {
+      const float4 q = *reinterpret_cast<const float4*>(p.params + e[i][0]);
+      w[i][0] = q.x; w[i][1] = q.y; w[i][2] = q.z; w[i][3] = q.w;
+      if constexpr (OPT != SEG_SGD) {
+        const float4 t = *reinterpret_cast<const float4*>(p.s1 + e[i][0]);
+        m[i][0] = t.x; m[i][1] = t.y; m[i][2] = t.z; m[i][3] = t.w;
+      }
+      if constexpr (OPT == SEG_ADAM) {
+        const float4 t = *reinterpret_cast<const float4*>(p.s2 + e[i][0]);
+        v[i][0] = t.x; v[i][1] = t.y; v[i][2] = t.z; v[i][3] = t.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (e[i][j] < 0) continue;
         w[i][j] = p.params[e[i][j]];
         if constexpr (OPT != SEG_SGD) m[i][j] = p.s1[e[i][j]];
         if constexpr (OPT == SEG_ADAM) v[i][j] = p.s2[e[i][j]];
@@ -478,14 +513,22 @@ small_wgrad_update_kernel(SmallStep p, int splits, int k_per_split) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (e[i][j] < 0) continue;
-      const float g = acc[i][j];
-      opt_step<OPT>(w[i][j], g, m[i][j], v[i][j], p, inv_bc1, inv_bc2);
-      p.grads[e[i][j]] = g;
-      if constexpr (OPT != SEG_SGD) p.s1[e[i][j]] = m[i][j];
-      if constexpr (OPT == SEG_ADAM) p.s2[e[i][j]] = v[i][j];
-      p.params[e[i][j]] = w[i][j];
+    for (int j = 0; j < 4; ++j)
+      if (e[i][j] >= 0) opt_step<OPT>(w[i][j], acc[i][j], m[i][j], v[i][j], p, inv_bc1, inv_bc2);
+    if (wide[i]) {
+      *reinterpret_cast<float4*>(p.grads + e[i][0]) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+      if constexpr (OPT != SEG_SGD) *reinterpret_cast<float4*>(p.s1 + e[i][0]) = make_float4(m[i][0], m[i][1], m[i][2], m[i][3]);
+      if constexpr (OPT == SEG_ADAM) *reinterpret_cast<float4*>(p.s2 + e[i][0]) = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+      *reinterpret_cast<float4*>(p.params + e[i][0]) = make_float4(w[i][0], w[i][1], w[i][2], w[i][3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (e[i][j] < 0) continue;
+        p.grads[e[i][j]] = acc[i][j];
+        if constexpr (OPT != SEG_SGD) p.s1[e[i][j]] = m[i][j];
+        if constexpr (OPT == SEG_ADAM) p.s2[e[i][j]] = v[i][j];
+        p.params[e[i][j]] = w[i][j];
+      }
     }
   }
 }
