@@ -32,8 +32,11 @@ def test_tensor_core_cases_with_forced_kernel_selection(env):
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-1000:]
 
 
-def test_fp32_cases_launch_by_launch():
-    child_env = dict(os.environ, SEG_NO_SMALL_FUSED="1")
+@pytest.mark.parametrize("env", [{"SEG_NO_SMALL_FUSED": "1"}, {"SEG_NO_GRAPH": "1"}, {"SEG_NO_PDL": "1"}])
+def test_fp32_cases_with_switches(env):
+    """The fp32 cases once more: launch by launch (no two-launch step for small segments), and the two-launch step
+    without the captured graph and without programmatic dependent launches."""
+    child_env = dict(os.environ, **env)
     res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-m", "gpu", "-q", "-x",
                           "-k", "fp32 or tiny or reproducible or replayed or class_index"], cwd=ROOT, env=child_env,
                          capture_output=True, text=True, timeout=900)
